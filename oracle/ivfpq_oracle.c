@@ -1,0 +1,243 @@
+/*
+ * CPU oracle for the sparsity-aware IVFPQ query path.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow restatement of what the path computes, written from the paper and
+ * used only by the tests, by the smoke check and by the benchmark's CPU-baseline
+ * leg.  It shares no code with the CUDA library and the product never calls it.
+ *
+ * Arithmetic: fp32, round to nearest, no contraction other than the explicit
+ * fmaf() calls (compile with -ffp-contract=off and without -ffast-math).  The
+ * paper does not state a precision; fp32 is this repository's reading.
+ *
+ * Steps (one query at a time; OpenMP only spreads independent queries):
+ *   S1  filtering: squared L2 distance from the query to every IVF centroid, the
+ *       nprobe closest are kept (Sec. 2.1 "Online Search", step A; Eq. "metric").
+ *   S2  selective L2-LUT: for every probed cluster the residual query - centroid;
+ *       in every subspace the squared distance from the residual projection to each
+ *       codebook entry; an entry is selected when that distance is within the
+ *       threshold radius of the subspace (Sec. 2.1 steps B, C; Sec. 3.1 "Intuition of
+ *       Algorithm Enhancement" and the last sentence of "Determining Proper
+ *       Threshold"; Algorithm 2, whose ray test against a sphere of radius
+ *       thres*thres_scale decides exactly d <= thres*thres_scale).  The table holds
+ *       the squared distance: only that makes the sum over subspaces the distance
+ *       of step D.
+ *   S3  distance calculation: every point of a probed cluster sums the table values
+ *       of its codes over the subspaces in which its entry was selected (step D);
+ *       each subspace whose entry was not selected contributes the large constant P
+ *       instead of a table look-up (Sec. 4.3, paragraph after Algorithm 2).
+ *   S4  the k smallest (distance, id) pairs, ascending (Sec. 2.1, last paragraph).
+ * Dense search is the same with every entry selected.
+ *
+ * Parity pins (tests/test_oracle_pins.py): radius -> inf equals dense bit for bit;
+ * dense distance equals the fp64 distance to the reconstructed vector; a lossless
+ * toy index reproduces brute-force exact neighbours; nesting/monotonicity in radius
+ * and nprobe; a naive second implementation without any table; the ray-time
+ * algebra of Algorithm 2 against the plain compare.  The paper's absolute recall
+ * and throughput figures are not recoverable from its text: parity unpinned
+ * against those, everything computed here is pinned by the tests above.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    float dist;
+    int32_t id;
+} cand_t;
+
+static int cand_less(const void* a, const void* b) {
+    const cand_t* x = (const cand_t*)a;
+    const cand_t* y = (const cand_t*)b;
+    if (x->dist < y->dist) return -1;
+    if (x->dist > y->dist) return 1;
+    if (x->id < y->id) return -1;
+    if (x->id > y->id) return 1;
+    return 0;
+}
+
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_num_threads(int n) {
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
+/* S1 for one query: dc[c] for all centroids, then the nprobe smallest by (dc, c). */
+static void coarse_one(const float* q, int d, const float* cent, int nlist, int nprobe,
+                       cand_t* scratch, int32_t* probe_ids, float* probe_d) {
+    for (int c = 0; c < nlist; ++c) {
+        float a = 0.0f;
+        for (int j = 0; j < d; ++j) {
+            float t = q[j] - cent[(size_t)c * d + j];
+            a = fmaf(t, t, a);
+        }
+        scratch[c].dist = a;
+        scratch[c].id = c;
+    }
+    qsort(scratch, (size_t)nlist, sizeof(cand_t), cand_less);
+    for (int p = 0; p < nprobe; ++p) {
+        probe_ids[p] = scratch[p].id;
+        probe_d[p] = scratch[p].dist;
+    }
+}
+
+int oracle_coarse(const float* queries, int64_t nq, int d, const float* cent, int nlist, int nprobe,
+                  int32_t* probe_ids, float* probe_d) {
+    if (nprobe > nlist || nprobe <= 0) return -1;
+#pragma omp parallel
+    {
+        cand_t* scratch = (cand_t*)malloc(sizeof(cand_t) * (size_t)nlist);
+#pragma omp for schedule(dynamic, 4)
+        for (int64_t qi = 0; qi < nq; ++qi)
+            coarse_one(queries + qi * d, d, cent, nlist, nprobe, scratch, probe_ids + qi * nprobe,
+                       probe_d + qi * nprobe);
+        free(scratch);
+    }
+    return 0;
+}
+
+/*
+ * Full search.  dense != 0 ignores the radius arguments.
+ *   radius       : mode 0 -> [nsub], mode 1 -> [nq][nsub]   (threshold before scaling)
+ *   scale        : the user scaling factor (thres_scale of Algorithm 2)
+ *   miss_penalty : P; negative -> P = sum over subspaces of the squared scaled radius
+ * Optional stage dumps (NULL to skip):
+ *   probe_ids/probe_d [nq][nprobe]; masks [nq][nprobe][nsub][8] (bit e of the 256-bit
+ *   row = entry e selected); visit_count [nq]; and, with visit_stride slots per query in
+ *   visiting order (probe rank, then position in the list): visit_hits (bit s = subspace
+ *   s selected for that point), visit_dist, visit_ids.
+ */
+int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* cent,
+                  const float* codebooks, const int64_t* list_offsets, const uint8_t* codes,
+                  const int32_t* ids, const float* queries, int64_t nq, int nprobe, int dense,
+                  const float* radius, int radius_mode, float scale, float miss_penalty, int k,
+                  float* out_dist, int32_t* out_ids, int32_t* probe_ids_out, float* probe_d_out,
+                  uint32_t* masks_out, int64_t* visit_count, int64_t visit_stride,
+                  uint64_t* visit_hits, float* visit_dist, int32_t* visit_ids) {
+    if (d != nsub * dsub || ksub <= 0 || ksub > 256 || nsub > 64) return -2;
+    if (nprobe <= 0 || nprobe > nlist || k <= 0) return -1;
+    if (!dense && radius == NULL) return -1;
+    int status = 0;
+
+#pragma omp parallel
+    {
+        cand_t* scratch = (cand_t*)malloc(sizeof(cand_t) * (size_t)nlist);
+        int32_t* probes = (int32_t*)malloc(sizeof(int32_t) * (size_t)nprobe);
+        float* probes_d = (float*)malloc(sizeof(float) * (size_t)nprobe);
+        float* lut = (float*)malloc(sizeof(float) * (size_t)nsub * ksub);
+        uint8_t* hit = (uint8_t*)malloc((size_t)nsub * ksub);
+        float* r2 = (float*)malloc(sizeof(float) * (size_t)nsub);
+        size_t cap = 1024, n = 0;
+        cand_t* vis = (cand_t*)malloc(sizeof(cand_t) * cap);
+
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t qi = 0; qi < nq; ++qi) {
+            const float* q = queries + qi * d;
+            coarse_one(q, d, cent, nlist, nprobe, scratch, probes, probes_d);
+            if (probe_ids_out) memcpy(probe_ids_out + qi * nprobe, probes, sizeof(int32_t) * nprobe);
+            if (probe_d_out) memcpy(probe_d_out + qi * nprobe, probes_d, sizeof(float) * nprobe);
+
+            /* threshold per (query, subspace), independent of the probed cluster */
+            float P = 0.0f;
+            if (!dense) {
+                const float* rad = radius_mode == 1 ? radius + qi * nsub : radius;
+                float acc = 0.0f;
+                for (int s = 0; s < nsub; ++s) {
+                    float r = rad[s] * scale;
+                    r2[s] = r * r;
+                    acc = acc + r2[s];
+                }
+                P = miss_penalty >= 0.0f ? miss_penalty : acc;
+            }
+
+            n = 0;
+            int64_t nvis = 0;
+            for (int p = 0; p < nprobe; ++p) {
+                const int c = probes[p];
+                /* S2: table and selection for this (query, cluster) */
+                for (int s = 0; s < nsub; ++s) {
+                    uint32_t mrow[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                    for (int e = 0; e < ksub; ++e) {
+                        const float* entry = codebooks + ((size_t)s * ksub + e) * dsub;
+                        float d2 = 0.0f;
+                        for (int j = 0; j < dsub; ++j) {
+                            float res = q[s * dsub + j] - cent[(size_t)c * d + s * dsub + j];
+                            float t = res - entry[j];
+                            d2 = fmaf(t, t, d2);
+                        }
+                        int h = dense ? 1 : (d2 <= r2[s]);
+                        lut[(size_t)s * ksub + e] = d2;
+                        hit[(size_t)s * ksub + e] = (uint8_t)h;
+                        if (h) mrow[e >> 5] |= 1u << (e & 31);
+                    }
+                    if (masks_out)
+                        memcpy(masks_out + (((size_t)qi * nprobe + p) * nsub + s) * 8, mrow, sizeof(mrow));
+                }
+                /* S3: every point of the cluster */
+                for (int64_t x = list_offsets[c]; x < list_offsets[c + 1]; ++x) {
+                    const uint8_t* code = codes + (size_t)x * nsub;
+                    float S = 0.0f;
+                    int m = 0;
+                    uint64_t hs = 0;
+                    for (int s = 0; s < nsub; ++s) {
+                        int e = code[s];
+                        if (e < ksub && hit[(size_t)s * ksub + e]) {
+                            S = S + lut[(size_t)s * ksub + e];
+                            hs |= (uint64_t)1 << s;
+                        } else {
+                            m += 1;
+                        }
+                    }
+                    float dist = (m == 0) ? S : fmaf((float)m, P, S);
+                    if (n == cap) {
+                        cap *= 2;
+                        vis = (cand_t*)realloc(vis, sizeof(cand_t) * cap);
+                    }
+                    vis[n].dist = dist;
+                    vis[n].id = ids[x];
+                    ++n;
+                    if (nvis < visit_stride) {
+                        if (visit_hits) visit_hits[qi * visit_stride + nvis] = hs;
+                        if (visit_dist) visit_dist[qi * visit_stride + nvis] = dist;
+                        if (visit_ids) visit_ids[qi * visit_stride + nvis] = ids[x];
+                    }
+                    ++nvis;
+                }
+            }
+            if (visit_count) visit_count[qi] = nvis;
+
+            /* S4 */
+            qsort(vis, n, sizeof(cand_t), cand_less);
+            for (int i = 0; i < k; ++i) {
+                if ((size_t)i < n) {
+                    out_dist[qi * k + i] = vis[i].dist;
+                    out_ids[qi * k + i] = vis[i].id;
+                } else {
+                    out_dist[qi * k + i] = INFINITY;
+                    out_ids[qi * k + i] = -1;
+                }
+            }
+        }
+        free(vis);
+        free(r2);
+        free(hit);
+        free(lut);
+        free(probes_d);
+        free(probes);
+        free(scratch);
+    }
+    return status;
+}
