@@ -1,0 +1,163 @@
+/*
+ * ivfpq.h - C ABI of the B200 (sm_100a) sparsity-aware IVFPQ query library.
+ *
+ * The library runs the online search phase of an IVFPQ index on one GPU:
+ *   (1) filtering: squared-L2 distances from each query to the IVF centroids, the nprobe
+ *       closest clusters are kept (paper Sec. 2.1 "Online Search", step A);
+ *   (2) L2-LUT construction for every (query, probed cluster): residual = query - centroid,
+ *       squared distance from each residual projection to each codebook entry (steps B, C);
+ *       in the sparsity-aware search only the entries within the threshold radius of the
+ *       projection are selected (Sec. 3.1; Algorithm 2, whose ray/sphere test decides exactly
+ *       "distance <= thres * thres_scale");
+ *   (3) distance calculation: every point of a probed cluster accumulates the table values of
+ *       its codes; a subspace whose entry was not selected contributes the large constant P
+ *       instead (Sec. 2.1 step D; Sec. 4.3, paragraph after Algorithm 2); then the k
+ *       smallest (distance, id) pairs per query (Sec. 2.1, last paragraph).
+ *
+ * Naming: nsub = number of PQ subspaces (the paper's D/M), dsub = dimensions per subspace (the
+ * paper's M), ksub = entries per codebook (the paper's E, at most 256: codes are bytes),
+ * nlist = IVF clusters (C), nprobe = probed clusters per query (nprobs).
+ * All distances are SQUARED L2 (Eq. "metric").  All floating point is fp32.
+ *
+ * Conventions for every entry point:
+ *   - returns IVFPQ_OK (0) or a negative IVFPQ_ERR_* code; never throws, never aborts;
+ *   - "dev" pointers are device memory owned by the caller (e.g. torch tensors) that must stay
+ *     alive until the work enqueued on `stream` has finished; "host" pointers are host memory;
+ *   - the library allocates no device memory (except where an entry point says otherwise): index
+ *     arrays, derived tables, workspace, queries and outputs all belong to the caller;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream); calls are
+ *     asynchronous on it unless stated otherwise;
+ *   - there is no CPU fallback: without a CUDA device every compute call fails with IVFPQ_ERR_CUDA.
+ */
+#ifndef IVFPQ_H
+#define IVFPQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define IVFPQ_OK 0
+#define IVFPQ_ERR_INVALID_ARGUMENT (-1) /* null pointer, non-positive size, bad offsets        */
+#define IVFPQ_ERR_UNSUPPORTED (-2)      /* ksub > 256, nsub > 64, dsub > 16, k > 1024, nprobe > nlist ... */
+#define IVFPQ_ERR_WORKSPACE (-3)        /* workspace or derived buffer too small / misaligned     */
+#define IVFPQ_ERR_CUDA (-4)             /* a CUDA runtime call or kernel launch failed            */
+#define IVFPQ_ERR_DEVICE_FLAG (-5)      /* a kernel raised its bounds / bounded-wait error flag   */
+
+#define IVFPQ_MAX_K 1024
+#define IVFPQ_MAX_NPROBE 1024
+#define IVFPQ_MAX_NSUB 64
+#define IVFPQ_MAX_DSUB 16
+
+typedef struct ivfpq_index ivfpq_index_t; /* opaque host-side handle */
+
+/* Description of a trained, encoded index (the conventional IVFPQ offline phase, Sec. 2.1 /
+ * Algorithm 1 without the ray-tracing scene and without the entry->points map). */
+typedef struct {
+    int32_t d;      /* vector dimension, = nsub * dsub                                   */
+    int32_t nlist;  /* IVF clusters                                                      */
+    int32_t nsub;   /* PQ subspaces, 1..64                                               */
+    int32_t dsub;   /* dimensions per subspace, 1..16                                    */
+    int32_t ksub;   /* entries per codebook, 1..256                                      */
+    int32_t metric; /* 0 = squared L2 (the only one supported)                           */
+    int64_t ntotal; /* encoded points                                                    */
+    const float* coarse_centroids; /* dev  [nlist][d]                                    */
+    const float* codebooks;        /* dev  [nsub][ksub][dsub], trained on residuals      */
+    const int64_t* list_offsets;   /* HOST [nlist+1], CSR offsets into codes/ids; copied */
+    const uint8_t* codes;          /* dev  [ntotal][nsub], list-contiguous               */
+    const int32_t* ids;            /* dev  [ntotal], list-contiguous, original ids >= 0  */
+} ivfpq_index_desc_t;
+
+/* Bytes of caller-owned device memory that ivfpq_index_load needs for derived tables (codes
+ * re-laid-out in 32-point interleaved blocks, list tables).  0 on invalid descriptions. */
+size_t ivfpq_index_derived_bytes(const ivfpq_index_desc_t* desc);
+
+/* Validates the description, builds the derived tables in `derived_dev` (256-byte aligned, at
+ * least ivfpq_index_derived_bytes) with kernels enqueued on `stream`, and returns a handle.
+ * After the stream work completes the search path reads coarse_centroids, codebooks, ids and
+ * derived_dev, but no longer desc->codes.  The handle itself is host memory owned by the
+ * library until ivfpq_index_free. */
+int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t derived_bytes,
+                     void* stream, ivfpq_index_t** out);
+int ivfpq_index_free(ivfpq_index_t* index);
+
+/* Radius parameters of the sparsity-aware search.  The threshold of subspace s for query q is
+ * radius[s] (mode 0) or radius[q*nsub + s] (mode 1), times `scale` (the user scaling factor,
+ * thres_scale in Algorithm 2); an entry is selected when its squared distance to the residual
+ * projection is <= (radius*scale)^2.  miss_penalty is the constant P added per subspace whose
+ * entry was not selected; a negative value asks for the default P = sum over subspaces of
+ * (radius*scale)^2 of that query, which ranks points first by number of missed subspaces. */
+typedef struct {
+    const float* radius; /* dev; mode 0: [nsub], mode 1: [nq][nsub] */
+    int32_t mode;
+    float scale;
+    float miss_penalty;
+} ivfpq_radius_t;
+
+/* Workspace (dev, 256-byte aligned) needed by one search call of this shape. */
+size_t ivfpq_search_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k);
+
+/* Conventional (dense) IVFPQ search: every codebook entry is selected.
+ * queries dev [nq][d]; out_dist dev [nq][k] ascending; out_ids dev [nq][k]; ties are ordered by
+ * ascending id; when fewer than k points were visited the tail is (+inf, -1). */
+int ivfpq_search_dense(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                       int32_t k, float* out_dist, int32_t* out_ids, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
+/* Sparsity-aware search (threshold-based selective L2-LUT, Sec. 3.1 / Algorithm 2, followed
+ * by the distance calculation of Sec. 4.3).  Same outputs as the dense search. */
+int ivfpq_search_sparse(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                        const ivfpq_radius_t* radius, int32_t k, float* out_dist, int32_t* out_ids,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* End-to-end variants with HOST query and result buffers (pinned memory recommended): copy the
+ * queries to the device, search, copy distances and ids back, all enqueued on `stream`.  The
+ * staging areas live in the caller's workspace, whose size is given by
+ * ivfpq_search_host_workspace_bytes.  `radius` (NULL = dense search) still points to a struct
+ * whose `radius` array is device memory. */
+size_t ivfpq_search_host_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k);
+int ivfpq_search_host(const ivfpq_index_t* index, const float* queries_host, int64_t nq, int32_t nprobe,
+                      const ivfpq_radius_t* radius, int32_t k, float* out_dist_host,
+                      int32_t* out_ids_host, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream` and reports the device-side status word of the last search that used
+ * `workspace`: IVFPQ_OK, IVFPQ_ERR_DEVICE_FLAG (a kernel found an out-of-range list id, code
+ * block or candidate count and skipped the access) or IVFPQ_ERR_CUDA. */
+int ivfpq_sync_status(const ivfpq_index_t* index, void* workspace, void* stream);
+
+/* Tuning knobs (host-side state of the handle; not thread-safe against concurrent searches).
+ *   IVFPQ_OPT_NSPLIT: number of CTAs that share one query's probe list (0 = automatic:
+ *   1 for large batches, more when nq alone cannot fill the GPU).  Results do not depend on it. */
+#define IVFPQ_OPT_NSPLIT 1
+int ivfpq_index_set_option(ivfpq_index_t* index, int32_t option, int64_t value);
+
+/* Number of kernel launches the most recent search call on this handle enqueued. */
+int64_t ivfpq_last_launch_count(const ivfpq_index_t* index);
+
+const char* ivfpq_error_string(int code);
+
+/* ---- test-only exports (small inputs) -------------------------------------------------------
+ * ivfpq_debug_probes: filtering stage alone. probe_ids dev [nq][nprobe] (ascending distance, ties
+ * by ascending cluster id), probe_d dev [nq][nprobe].
+ *
+ * ivfpq_debug_search: the production kernels compiled with stage dumps.  radius NULL = dense.
+ * Any dump pointer may be NULL.  masks dev [nq][nprobe][nsub][8] (bit e of the 256-bit row =
+ * entry e selected); visit_* dev [nq][visit_stride] in visiting order (probe rank, then position
+ * in the list): visit_hits bit s = subspace s selected for that point, visit_dist its
+ * accumulated distance, visit_ids its id; visit_count dev [nq] int64.  Uses workspace of
+ * ivfpq_search_workspace_bytes. */
+int ivfpq_debug_probes(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                       int32_t* probe_ids, float* probe_d, void* workspace, size_t workspace_bytes,
+                       void* stream);
+int ivfpq_debug_search(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                       const ivfpq_radius_t* radius, int32_t k, float* out_dist, int32_t* out_ids,
+                       int32_t* probe_ids, float* probe_d, uint32_t* masks, int64_t* visit_count,
+                       int64_t visit_stride, uint64_t* visit_hits, float* visit_dist,
+                       int32_t* visit_ids, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IVFPQ_H */

@@ -1,0 +1,391 @@
+// C ABI of the IVFPQ query library: argument validation, workspace carve-up, kernel sequencing.
+// See include/ivfpq.h for the contract of every entry point.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace ivfpq {
+
+namespace {
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+struct DerivedLayout {
+    size_t list_off_off, list_blk_off, codes_off, total;
+    int64_t nblocks, max_len;
+    int32_t nw, vec16;
+};
+
+// Validates the description and lays out the derived buffer.  Returns an IVFPQ_* code.
+int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
+    if (!d) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (d->d <= 0 || d->nlist <= 0 || d->nsub <= 0 || d->dsub <= 0 || d->ksub <= 0 || d->ntotal < 0)
+        return IVFPQ_ERR_INVALID_ARGUMENT;
+    if ((int64_t)d->nsub * d->dsub != d->d) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (d->metric != 0 || d->ksub > 256 || d->nsub > IVFPQ_MAX_NSUB || d->dsub > IVFPQ_MAX_DSUB)
+        return IVFPQ_ERR_UNSUPPORTED;
+    if (d->ntotal > 0x7FFFFFFFll) return IVFPQ_ERR_UNSUPPORTED;  // ids are int32
+    if (!d->list_offsets) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (d->list_offsets[0] != 0 || d->list_offsets[d->nlist] != d->ntotal) return IVFPQ_ERR_INVALID_ARGUMENT;
+    int64_t nblocks = 0, max_len = 0;
+    for (int c = 0; c < d->nlist; ++c) {
+        const int64_t len = d->list_offsets[c + 1] - d->list_offsets[c];
+        if (len < 0) return IVFPQ_ERR_INVALID_ARGUMENT;
+        nblocks += (len + kPointsPerBlock - 1) / kPointsPerBlock;
+        if (len > max_len) max_len = len;
+    }
+    out->nw = (d->nsub + 3) / 4;
+    out->vec16 = (out->nw % 4 == 0) ? 1 : 0;
+    out->nblocks = nblocks;
+    out->max_len = max_len;
+    size_t off = 0;
+    out->list_off_off = off;
+    off = align_up(off + sizeof(int64_t) * (size_t)(d->nlist + 1), 256);
+    out->list_blk_off = off;
+    off = align_up(off + sizeof(int64_t) * (size_t)(d->nlist + 1), 256);
+    out->codes_off = off;
+    off = align_up(off + (size_t)nblocks * kPointsPerBlock * out->nw * 4, 256);
+    out->total = off > 0 ? off : 256;
+    return IVFPQ_OK;
+}
+
+int check_search_shape(const ivfpq_index* ix, int64_t nq, int32_t nprobe, int32_t k) {
+    if (!ix) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (nq <= 0 || nprobe <= 0 || k <= 0) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (nprobe > ix->nlist || nprobe > IVFPQ_MAX_NPROBE || k > IVFPQ_MAX_K) return IVFPQ_ERR_UNSUPPORTED;
+    if (nq > (int64_t)1 << 24) return IVFPQ_ERR_UNSUPPORTED;
+    return IVFPQ_OK;
+}
+
+int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stream, bool probes_only) {
+    const ivfpq_index* ix = a.ix;
+    int rc = check_search_shape(ix, a.nq, a.nprobe, a.k);
+    if (rc != IVFPQ_OK) return rc;
+    if (!a.queries || !workspace) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (!probes_only && (!a.out_dist || !a.out_ids)) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (!a.dense) {
+        if (!a.radius || (a.radius_mode != 0 && a.radius_mode != 1)) return IVFPQ_ERR_INVALID_ARGUMENT;
+        if (isnan(a.scale) || isnan(a.miss_penalty)) return IVFPQ_ERR_INVALID_ARGUMENT;
+    }
+    if (!aligned(a.queries, 4) || !aligned(workspace, 256)) return IVFPQ_ERR_WORKSPACE;
+    const WorkspaceLayout wl = plan_workspace(ix, a.nq, a.nprobe, a.k);
+    if (workspace_bytes < wl.total) return IVFPQ_ERR_WORKSPACE;
+
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    int64_t launches = 0;
+    if (cudaMemsetAsync(ws + wl.status_off, 0, 16, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    int32_t* probe_ids = reinterpret_cast<int32_t*>(ws + wl.probe_ids_off);
+    float* probe_d = reinterpret_cast<float*>(ws + wl.probe_d_off);
+    if (launch_coarse(ix, a.queries, a.nq, a.nprobe, reinterpret_cast<float*>(ws + wl.coarse_off), wl.qchunk,
+                      probe_ids, probe_d, reinterpret_cast<int*>(ws + wl.status_off), st, &launches) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    const size_t pbytes = (size_t)a.nq * a.nprobe * 4;
+    if (a.probe_ids_out &&
+        cudaMemcpyAsync(a.probe_ids_out, probe_ids, pbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    if (a.probe_d_out && cudaMemcpyAsync(a.probe_d_out, probe_d, pbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    if (!probes_only) {
+        if (launch_scan(a, wl, ws, st, &launches) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    }
+    ix->last_launches = launches;
+    return IVFPQ_OK;
+}
+
+}  // namespace
+
+WorkspaceLayout plan_workspace(const ivfpq_index* ix, int64_t nq, int32_t nprobe, int32_t k) {
+    WorkspaceLayout wl{};
+    // query chunk of the filtering stage: keep the [qchunk][nlist] distance tile near 32 MiB so
+    // that it stays in L2 between the kernel that writes it and the one that selects from it
+    int64_t qchunk = ((int64_t)32 << 20) / ((int64_t)ix->nlist * 4);
+    if (qchunk < 64) qchunk = 64;
+    if (qchunk > nq) qchunk = nq;
+    wl.qchunk = qchunk;
+    int nsplit = ix->nsplit_opt;
+    if (nsplit <= 0) {
+        // enough CTAs for two waves of the device at 4 CTAs per SM
+        const int64_t want = (int64_t)ix->sm_count * 8;
+        nsplit = (int)((want + nq - 1) / nq);
+        if (nsplit < 1) nsplit = 1;
+    }
+    if (nsplit > nprobe) nsplit = nprobe;
+    if (nsplit > 64) nsplit = 64;
+    wl.nsplit = nsplit;
+    size_t off = 0;
+    wl.status_off = off;
+    off = align_up(off + 16, 256);
+    wl.probe_ids_off = off;
+    off = align_up(off + (size_t)nq * nprobe * 4, 256);
+    wl.probe_d_off = off;
+    off = align_up(off + (size_t)nq * nprobe * 4, 256);
+    wl.coarse_off = off;
+    off = align_up(off + (size_t)qchunk * ix->nlist * 4, 256);
+    wl.partial_off = off;
+    // sized for the largest split the option may select later, so that the option can change
+    // without a new workspace query
+    off = align_up(off + (size_t)nq * (size_t)(nprobe < 64 ? nprobe : 64) * k * 8, 256);
+    wl.total = off;
+    return wl;
+}
+
+}  // namespace ivfpq
+
+using namespace ivfpq;
+
+extern "C" {
+
+size_t ivfpq_index_derived_bytes(const ivfpq_index_desc_t* desc) {
+    DerivedLayout dl;
+    if (plan_derived(desc, &dl) != IVFPQ_OK) return 0;
+    return dl.total;
+}
+
+int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t derived_bytes, void* stream,
+                     ivfpq_index_t** out) {
+    if (!out) return IVFPQ_ERR_INVALID_ARGUMENT;
+    *out = nullptr;
+    DerivedLayout dl;
+    int rc = plan_derived(desc, &dl);
+    if (rc != IVFPQ_OK) return rc;
+    if (!desc->coarse_centroids || !desc->codebooks || !derived_dev) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (desc->ntotal > 0 && (!desc->codes || !desc->ids)) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (!aligned(derived_dev, 256) || derived_bytes < dl.total) return IVFPQ_ERR_WORKSPACE;
+    if (!aligned(desc->coarse_centroids, 16) || !aligned(desc->codebooks, 16) || !aligned(desc->ids, 4))
+        return IVFPQ_ERR_INVALID_ARGUMENT;
+
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return IVFPQ_ERR_CUDA;
+
+    ivfpq_index* ix = new (std::nothrow) ivfpq_index();
+    if (!ix) return IVFPQ_ERR_INVALID_ARGUMENT;
+    ix->d = desc->d;
+    ix->nlist = desc->nlist;
+    ix->nsub = desc->nsub;
+    ix->dsub = desc->dsub;
+    ix->ksub = desc->ksub;
+    ix->ntotal = desc->ntotal;
+    ix->cent = desc->coarse_centroids;
+    ix->cb = desc->codebooks;
+    ix->ids = desc->ids;
+    char* base = static_cast<char*>(derived_dev);
+    ix->list_off = reinterpret_cast<const int64_t*>(base + dl.list_off_off);
+    ix->list_blk = reinterpret_cast<const int64_t*>(base + dl.list_blk_off);
+    ix->codes_il = reinterpret_cast<const uint32_t*>(base + dl.codes_off);
+    ix->nw = dl.nw;
+    ix->vec16 = dl.vec16;
+    ix->nblocks = dl.nblocks;
+    ix->max_list_len = dl.max_len;
+    ix->device = dev;
+    ix->sm_count = sms;
+    ix->nsplit_opt = 0;
+    ix->last_launches = 0;
+
+    // list tables: built on the host, copied synchronously (pageable source)
+    const size_t n1 = (size_t)desc->nlist + 1;
+    int64_t* blk = new (std::nothrow) int64_t[n1];
+    if (!blk) {
+        delete ix;
+        return IVFPQ_ERR_INVALID_ARGUMENT;
+    }
+    blk[0] = 0;
+    for (int c = 0; c < desc->nlist; ++c) {
+        const int64_t len = desc->list_offsets[c + 1] - desc->list_offsets[c];
+        blk[c + 1] = blk[c] + (len + kPointsPerBlock - 1) / kPointsPerBlock;
+    }
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(base + dl.list_off_off, desc->list_offsets, n1 * 8, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(base + dl.list_blk_off, blk, n1 * 8, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);  // the host arrays may go away after return
+    delete[] blk;
+    if (e == cudaSuccess)
+        e = launch_relayout(ix, desc->codes, reinterpret_cast<uint32_t*>(base + dl.codes_off), st);
+    if (e != cudaSuccess) {
+        delete ix;
+        return IVFPQ_ERR_CUDA;
+    }
+    *out = ix;
+    return IVFPQ_OK;
+}
+
+int ivfpq_index_free(ivfpq_index_t* index) {
+    if (!index) return IVFPQ_ERR_INVALID_ARGUMENT;
+    delete index;
+    return IVFPQ_OK;
+}
+
+size_t ivfpq_search_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k) {
+    if (check_search_shape(index, nq, nprobe, k) != IVFPQ_OK) return 0;
+    return plan_workspace(index, nq, nprobe, k).total;
+}
+
+int ivfpq_search_dense(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe, int32_t k,
+                       float* out_dist, int32_t* out_ids, void* workspace, size_t workspace_bytes, void* stream) {
+    SearchArgs a{};
+    a.ix = index;
+    a.queries = queries;
+    a.nq = nq;
+    a.nprobe = nprobe;
+    a.k = k;
+    a.dense = true;
+    a.out_dist = out_dist;
+    a.out_ids = out_ids;
+    return run_search(a, workspace, workspace_bytes, stream, false);
+}
+
+static void fill_radius(SearchArgs& a, const ivfpq_radius_t* radius) {
+    a.dense = false;
+    a.radius = radius->radius;
+    a.radius_mode = radius->mode;
+    a.scale = radius->scale;
+    a.miss_penalty = radius->miss_penalty;
+}
+
+int ivfpq_search_sparse(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                        const ivfpq_radius_t* radius, int32_t k, float* out_dist, int32_t* out_ids,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (!radius) return IVFPQ_ERR_INVALID_ARGUMENT;
+    SearchArgs a{};
+    a.ix = index;
+    a.queries = queries;
+    a.nq = nq;
+    a.nprobe = nprobe;
+    a.k = k;
+    fill_radius(a, radius);
+    a.out_dist = out_dist;
+    a.out_ids = out_ids;
+    return run_search(a, workspace, workspace_bytes, stream, false);
+}
+
+size_t ivfpq_search_host_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k) {
+    if (check_search_shape(index, nq, nprobe, k) != IVFPQ_OK) return 0;
+    size_t core = plan_workspace(index, nq, nprobe, k).total;
+    size_t off = align_up(core, 256);
+    off = align_up(off + (size_t)nq * index->d * 4, 256);
+    off = align_up(off + (size_t)nq * k * 4, 256);
+    off = align_up(off + (size_t)nq * k * 4, 256);
+    return off;
+}
+
+int ivfpq_search_host(const ivfpq_index_t* index, const float* queries_host, int64_t nq, int32_t nprobe,
+                      const ivfpq_radius_t* radius, int32_t k, float* out_dist_host, int32_t* out_ids_host,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_search_shape(index, nq, nprobe, k);
+    if (rc != IVFPQ_OK) return rc;
+    if (!queries_host || !out_dist_host || !out_ids_host || !workspace) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (!aligned(workspace, 256)) return IVFPQ_ERR_WORKSPACE;
+    if (workspace_bytes < ivfpq_search_host_workspace_bytes(index, nq, nprobe, k)) return IVFPQ_ERR_WORKSPACE;
+    const size_t core = align_up(plan_workspace(index, nq, nprobe, k).total, 256);
+    char* ws = static_cast<char*>(workspace);
+    size_t off = core;
+    float* q_dev = reinterpret_cast<float*>(ws + off);
+    off = align_up(off + (size_t)nq * index->d * 4, 256);
+    float* d_dev = reinterpret_cast<float*>(ws + off);
+    off = align_up(off + (size_t)nq * k * 4, 256);
+    int32_t* i_dev = reinterpret_cast<int32_t*>(ws + off);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(q_dev, queries_host, (size_t)nq * index->d * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    SearchArgs a{};
+    a.ix = index;
+    a.queries = q_dev;
+    a.nq = nq;
+    a.nprobe = nprobe;
+    a.k = k;
+    a.dense = true;
+    if (radius) fill_radius(a, radius);
+    a.out_dist = d_dev;
+    a.out_ids = i_dev;
+    rc = run_search(a, workspace, core, stream, false);
+    if (rc != IVFPQ_OK) return rc;
+    if (cudaMemcpyAsync(out_dist_host, d_dev, (size_t)nq * k * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    if (cudaMemcpyAsync(out_ids_host, i_dev, (size_t)nq * k * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    return IVFPQ_OK;
+}
+
+int ivfpq_sync_status(const ivfpq_index_t* index, void* workspace, void* stream) {
+    if (!index || !workspace) return IVFPQ_ERR_INVALID_ARGUMENT;
+    int flags[4] = {0, 0, 0, 0};
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(flags, workspace, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    return flags[0] != 0 ? IVFPQ_ERR_DEVICE_FLAG : IVFPQ_OK;
+}
+
+int ivfpq_index_set_option(ivfpq_index_t* index, int32_t option, int64_t value) {
+    if (!index) return IVFPQ_ERR_INVALID_ARGUMENT;
+    switch (option) {
+        case IVFPQ_OPT_NSPLIT:
+            if (value < 0 || value > 64) return IVFPQ_ERR_INVALID_ARGUMENT;
+            index->nsplit_opt = (int32_t)value;
+            return IVFPQ_OK;
+        default:
+            return IVFPQ_ERR_INVALID_ARGUMENT;
+    }
+}
+
+int64_t ivfpq_last_launch_count(const ivfpq_index_t* index) { return index ? index->last_launches : 0; }
+
+const char* ivfpq_error_string(int code) {
+    switch (code) {
+        case IVFPQ_OK: return "ok";
+        case IVFPQ_ERR_INVALID_ARGUMENT: return "invalid argument";
+        case IVFPQ_ERR_UNSUPPORTED: return "unsupported shape";
+        case IVFPQ_ERR_WORKSPACE: return "workspace or derived buffer too small or misaligned";
+        case IVFPQ_ERR_CUDA: return "CUDA runtime error";
+        case IVFPQ_ERR_DEVICE_FLAG: return "device-side status flag raised";
+        default: return "unknown error code";
+    }
+}
+
+int ivfpq_debug_probes(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                       int32_t* probe_ids, float* probe_d, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!probe_ids || !probe_d) return IVFPQ_ERR_INVALID_ARGUMENT;
+    SearchArgs a{};
+    a.ix = index;
+    a.queries = queries;
+    a.nq = nq;
+    a.nprobe = nprobe;
+    a.k = 1;
+    a.dense = true;
+    a.probe_ids_out = probe_ids;
+    a.probe_d_out = probe_d;
+    return run_search(a, workspace, workspace_bytes, stream, true);
+}
+
+int ivfpq_debug_search(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                       const ivfpq_radius_t* radius, int32_t k, float* out_dist, int32_t* out_ids,
+                       int32_t* probe_ids, float* probe_d, uint32_t* masks, int64_t* visit_count,
+                       int64_t visit_stride, uint64_t* visit_hits, float* visit_dist, int32_t* visit_ids,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    if (visit_stride < 0) return IVFPQ_ERR_INVALID_ARGUMENT;
+    SearchArgs a{};
+    a.ix = index;
+    a.queries = queries;
+    a.nq = nq;
+    a.nprobe = nprobe;
+    a.k = k;
+    a.dense = true;
+    if (radius) fill_radius(a, radius);
+    a.out_dist = out_dist;
+    a.out_ids = out_ids;
+    a.debug = true;
+    a.probe_ids_out = probe_ids;
+    a.probe_d_out = probe_d;
+    a.masks = masks;
+    a.visit_count = visit_count;
+    a.visit_stride = visit_stride;
+    a.visit_hits = visit_hits;
+    a.visit_dist = visit_dist;
+    a.visit_ids = visit_ids;
+    return run_search(a, workspace, workspace_bytes, stream, false);
+}
+
+}  // extern "C"

@@ -1,0 +1,94 @@
+// Internal declarations shared by the translation units of the IVFPQ library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ivfpq.h"
+
+namespace ivfpq {
+
+constexpr int kPointsPerBlock = 32;  // points per interleaved code block (one warp, one point per lane)
+constexpr int kScanThreads = 256;    // threads per scan CTA (= max entries per codebook)
+constexpr int kTopkCap = 2048;       // candidate buffer slots per CTA (>= IVFPQ_MAX_K + kScanThreads)
+
+// Device status bits (workspace status word).
+constexpr int kFlagBadList = 1;   // a probed cluster id or code block was out of range and was skipped
+constexpr int kFlagOverflow = 2;  // the candidate buffer would have overflowed; the candidate was dropped
+
+inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace ivfpq
+
+// Host-side handle.  All pointers are device pointers into caller-owned memory.
+struct ivfpq_index {
+    int32_t d, nlist, nsub, dsub, ksub;
+    int64_t ntotal;
+    const float* cent;        // [nlist][d]
+    const float* cb;          // [nsub][ksub][dsub]
+    const int32_t* ids;       // [ntotal] list-contiguous
+    // derived tables (inside the caller's derived buffer)
+    const int64_t* list_off;  // [nlist+1] point offsets (index into ids)
+    const int64_t* list_blk;  // [nlist+1] offsets in 32-point code blocks
+    const uint32_t* codes_il; // interleaved codes, see relayout.cu
+    int32_t nw;               // 4-byte code words per point (nsub rounded up to a multiple of 4)
+    int32_t vec16;            // 1: words grouped by four (16-byte lane loads), 0: single words
+    int64_t nblocks;          // total 32-point blocks
+    int64_t max_list_len;
+    // host state
+    int32_t device;
+    int32_t sm_count;
+    int32_t nsplit_opt;       // 0 = automatic
+    mutable int64_t last_launches;
+};
+
+namespace ivfpq {
+
+struct SearchArgs {
+    const ivfpq_index* ix;
+    const float* queries;     // dev [nq][d]
+    int64_t nq;
+    int32_t nprobe;
+    int32_t k;
+    bool dense;
+    const float* radius;      // dev
+    int32_t radius_mode;
+    float scale;
+    float miss_penalty;
+    float* out_dist;
+    int32_t* out_ids;
+    // dumps (debug build of the kernels), all optional
+    bool debug;
+    int32_t* probe_ids_out;
+    float* probe_d_out;
+    uint32_t* masks;
+    int64_t* visit_count;
+    int64_t visit_stride;
+    uint64_t* visit_hits;
+    float* visit_dist;
+    int32_t* visit_ids;
+};
+
+// Workspace carve-up (all offsets 256-byte aligned).
+struct WorkspaceLayout {
+    size_t status_off;      // 4 x int32
+    size_t probe_ids_off;   // [nq][nprobe] int32
+    size_t probe_d_off;     // [nq][nprobe] fp32
+    size_t coarse_off;      // [qchunk][nlist] fp32
+    size_t partial_off;     // [nq][nsplit][k] uint64 keys (nsplit > 1 only)
+    size_t total;
+    int64_t qchunk;
+    int32_t nsplit;
+};
+
+WorkspaceLayout plan_workspace(const ivfpq_index* ix, int64_t nq, int32_t nprobe, int32_t k);
+
+// Launchers (return cudaError_t of the launch; count launches into *launches).
+cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_t* codes_il, cudaStream_t st);
+cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,
+                          float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
+                          int* status, cudaStream_t st, int64_t* launches);
+cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws, cudaStream_t st,
+                        int64_t* launches);
+
+}  // namespace ivfpq
