@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the sparsity-aware IVFPQ query path on B200.
+
+One "step" is one pass of the whole hot path - filtering, selective L2-LUT
+construction, list scan, top-k - over one batch of synthetic queries through the C
+ABI (`ivfpq_search_sparse` at the radius scale whose recall@100 is within 0.01 of
+the dense search).  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--nprobe 16]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores
+
+Multi-GPU (torchrun, one rank per GPU): the index is replicated and every rank
+searches its own query batch - no data-path collective ("scaling": "weak").
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from ivfpq_inputs import CONFIGS, build_index_streamed, calibrate_radius, recall_1_at_k, recall_at_k  # noqa: E402
+from ivfpq_inputs import generators as G  # noqa: E402
+from ivfpq_inputs.groundtruth import ExactKnnAccumulator  # noqa: E402
+
+METRIC = "queries/sec at recall@100 (1 B200) + scan HBM GB/s as % of peak"
+UNIT = "queries/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one scan-kernel launch, from the ncu captures
+# summarised under profiles/ (bytes per launch of the benchmark's workload; None = not captured).
+SCAN_DRAM_TRAFFIC_BYTES = {}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {
+        0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x10: "sync_boost",
+        0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+        0x100: "display_clock_setting",
+    }
+
+    def __init__(self, device_index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        self._period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            uuid = torch.cuda.get_device_properties(device_index).uuid
+            try:
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # pragma: no cover
+            log(f"[bench] NVML unavailable: {e}")
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                for b, name in self.REASONS.items():
+                    if bits & b:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self._period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------
+# workload
+# --------------------------------------------------------------------------------------------
+
+def build_workload(name: str, device: str, nq: int | None, query_seed_offset: int = 0):
+    """Index + queries + exact neighbours + calibrated radii for one of the synthetic configs."""
+    cfg = CONFIGS[name]
+    if nq is not None:
+        cfg = cfg.scaled(nq=nq)
+    if query_seed_offset:
+        cfg = cfg.scaled(query_seed=cfg.query_seed + query_seed_offset)
+    t0 = time.time()
+    spec = G.make_mixture(cfg, device)
+    q = G.queries(cfg, spec)
+    acc = ExactKnnAccumulator(q, cfg.k)
+    index = build_index_streamed(cfg, spec, on_chunk=acc.add)
+    true_ids, _ = acc.result()
+    radius = calibrate_radius(index, G.calibration_queries(cfg, spec, 1000))
+    log(f"[bench] built {name}: N={index.ntotal} nlist={index.nlist} {index.nsub}x{index.dsub} "
+        f"nq={q.shape[0]} in {time.time() - t0:.1f}s on {device}")
+    return cfg, index, q.cpu().numpy(), true_ids, radius
+
+
+def pick_scale(search_sparse, search_dense, true_ids, scales=(0.5, 0.75, 1.0, 1.25, 1.5, 2.0, 3.0, 4.0)):
+    """Smallest radius scale whose recall@100 is within 0.01 of the dense search."""
+    dense_ids = search_dense()
+    r_dense = recall_at_k(dense_ids, true_ids)
+    table = []
+    chosen = None
+    for s in scales:
+        ids = search_sparse(s)
+        r = recall_at_k(ids, true_ids)
+        table.append((s, round(r, 4)))
+        if chosen is None and r >= r_dense - 0.01:
+            chosen = (s, r, recall_1_at_k(ids, true_ids))
+            break
+    if chosen is None:
+        ids = search_sparse(float("inf"))
+        chosen = (float("inf"), recall_at_k(ids, true_ids), recall_1_at_k(ids, true_ids))
+    return r_dense, recall_1_at_k(dense_ids, true_ids), chosen, table
+
+
+def visits_per_batch(index, probe_ids: np.ndarray) -> int:
+    lens = np.diff(index.list_offsets)
+    return int(lens[probe_ids].sum())
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------------------------
+
+def run_cuda(args):
+    import paper_2312_01712_b200 as lib
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("launch with torch.distributed.run for --gpus > 1")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback for the product path)")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    lib.load_library()
+    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq, query_seed_offset=rank)
+    nprobe = args.nprobe or cfg.nprobes[len(cfg.nprobes) // 2]
+    k = cfg.k
+    nq = q_np.shape[0]
+    h = lib.ivfpq_index_load(index, dev)
+    qd = torch.from_numpy(q_np).to(dev)
+    rad_d = torch.from_numpy(radius).to(dev)
+    out = (torch.empty((nq, k), dtype=torch.float32, device=dev), torch.empty((nq, k), dtype=torch.int32, device=dev))
+
+    def dense_ids():
+        return lib.ivfpq_search_dense(h, qd, nprobe, k)[1].cpu().numpy()
+
+    def sparse_ids(s):
+        return lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=s)[1].cpu().numpy()
+
+    r_dense, r1_dense, (scale, r_sparse, r1_sparse), sweep = pick_scale(sparse_ids, dense_ids, true_ids)
+    assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
+    log(f"[bench] recall@100 dense {r_dense:.4f}, sparse {r_sparse:.4f} at scale {scale} (sweep {sweep})")
+
+    probe_ids = lib.ivfpq_debug_probes(h, qd, nprobe)[0].cpu().numpy()
+    visits = visits_per_batch(index, probe_ids)
+    scan_bytes = visits * index.nsub          # algorithmic: one code byte per subspace per visited point
+
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
+    lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_TIMING, 1)
+
+    def step_sparse():
+        lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=scale, out=out)
+
+    def step_dense():
+        lib.ivfpq_search_dense(h, qd, nprobe, k, out=out)
+
+    def timed(step, steps, warmup, sampler=None, stage_acc=None):
+        for _ in range(warmup):
+            flush.zero_()
+            step()
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        ctx = sampler if sampler is not None else _Null()
+        with ctx:
+            for a, b in evs:
+                flush.zero_()            # L2 flush between timed iterations (not timed)
+                a.record()
+                step()
+                b.record()
+                if stage_acc is not None:
+                    stage_acc.append(lib.ivfpq_last_stage_ms(h))
+            torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        total_ms = sum(a.elapsed_time(b) for a, b in evs)
+        if dist is not None:
+            t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total_ms = float(t.item())
+        return total_ms
+
+    sampler = ClockSampler(local_rank)
+    stages = []
+    total_ms = timed(step_sparse, args.steps, args.warmup, sampler, stages)
+    launches = lib.ivfpq_last_launch_count(h) * args.steps
+    dense_ms = timed(step_dense, max(3, args.steps // 4), 3)
+    dense_steps = max(3, args.steps // 4)
+
+    # end to end: host buffers, copies inside the timed region
+    qh = torch.from_numpy(q_np).pin_memory()
+    odh = torch.empty((nq, k), dtype=torch.float32).pin_memory()
+    oih = torch.empty((nq, k), dtype=torch.int32).pin_memory()
+
+    def step_host():
+        lib.ivfpq_search_host(h, qh, nprobe, k, odh, oih, radius=rad_d, scale=scale)
+
+    lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_TIMING, 0)
+    e2e_steps = max(3, args.steps // 4)
+    e2e_ms = timed(step_host, e2e_steps, 3)
+    assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    scan_ms = float(np.mean([s[1] for s in stages]))
+    coarse_ms = float(np.mean([s[0] for s in stages]))
+    achieved = scan_bytes / (scan_ms * 1e-3) / 1e9
+
+    cpu = cpu_baseline(index, q_np, nprobe, k, radius, scale, args.cpu_sample)
+
+    line = {
+        "metric": METRIC, "value": nq * world * args.steps / (total_ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: N={index.ntotal} D={index.d} nlist={index.nlist} "
+                               f"PQ {index.nsub}x{index.dsub} (uint8 codes), nq={nq}/GPU, nprobe={nprobe}, k={k}, "
+                               f"sparse search at radius scale {scale}",
+                   "l2": "512 MiB buffer written between timed iterations (L2 flush)",
+                   "parallelism": "replicas only (index replicated, queries split)" if world > 1 else "1 GPU",
+                   "radius_scale": scale, "nprobe": nprobe},
+        "recall@100": {"sparse": round(r_sparse, 4), "dense": round(r_dense, 4),
+                       "R1@100_sparse": round(r1_sparse, 4), "R1@100_dense": round(r1_dense, 4)},
+        "dense_queries_per_s": nq * world * dense_steps / (dense_ms * 1e-3),
+        "sparse_over_dense": (dense_ms / dense_steps) / (total_ms / args.steps),
+        "stages_ms": {"filtering": round(coarse_ms, 4), "lut_scan_topk": round(scan_ms, 4)},
+        "e2e": {"value": nq * world * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": int(qh.numel() * 4), "d2h_bytes_per_step": int(odh.numel() * 4 + oih.numel() * 4)},
+        "gpu_launches": int(launches),
+        "clocks": sampler.summary(),
+        "roofline": {"bound": "hbm", "kernel": "scan_kernel (selective LUT + list scan + top-k)",
+                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_source": f"of {peak_src}", "algorithmic_bytes_per_launch": int(scan_bytes),
+                     "visits_per_launch": int(visits), "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload)},
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+class _Null:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        return False
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU oracle: cpu_baseline leg and --impl reference
+# --------------------------------------------------------------------------------------------
+
+def cpu_baseline(index, q_np, nprobe, k, radius, scale, sample):
+    import oracle
+    sample = min(sample, q_np.shape[0])
+    oracle.search(index, q_np[:8], nprobe, k, radius=radius, scale=scale)    # page in
+    t0 = time.perf_counter()
+    oracle.search(index, q_np[:sample], nprobe, k, radius=radius, scale=scale)
+    dt = time.perf_counter() - t0
+    return {"value": sample / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {sample} queries of the batch, one oracle.search call, {dt:.2f} s"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"      # input generation only
+    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq)
+    nprobe = args.nprobe or cfg.nprobes[len(cfg.nprobes) // 2]
+    k = cfg.k
+    sample = min(args.cpu_sample, q_np.shape[0])
+    scale = args.ref_scale
+    for _ in range(min(args.warmup, 1)):
+        oracle.search(index, q_np[:64], nprobe, k, radius=radius, scale=scale)
+    steps = min(args.steps, 5)
+    t0 = time.perf_counter()
+    for i in range(steps):
+        lo = (i * sample) % max(1, q_np.shape[0] - sample + 1)
+        oracle.search(index, q_np[lo:lo + sample], nprobe, k, radius=radius, scale=scale)
+    dt = time.perf_counter() - t0
+    value = sample * steps / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": dt / steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: N={index.ntotal} D={index.d} nlist={index.nlist} "
+                               f"PQ {index.nsub}x{index.dsub}, nprobe={nprobe}, k={k}, sparse search at radius "
+                               f"scale {scale}; each step = {sample} queries of the batch",
+                   "radius_scale": scale, "nprobe": nprobe},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": f"{steps} steps x {sample} queries"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(CONFIGS))
+    ap.add_argument("--nprobe", type=int, default=0)
+    ap.add_argument("--nq", type=int, default=None)
+    ap.add_argument("--cpu-sample", type=int, default=10000, help="queries timed on the CPU oracle")
+    ap.add_argument("--ref-scale", type=float, default=1.0)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "cuda":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

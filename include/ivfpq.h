@@ -131,7 +131,16 @@ int ivfpq_sync_status(const ivfpq_index_t* index, void* workspace, void* stream)
  *   IVFPQ_OPT_NSPLIT: number of CTAs that share one query's probe list (0 = automatic:
  *   1 for large batches, more when nq alone cannot fill the GPU).  Results do not depend on it. */
 #define IVFPQ_OPT_NSPLIT 1
+/*   IVFPQ_OPT_TIMING: 1 = record CUDA events around the filtering stage and around the
+ *   LUT+scan(+merge) stage of every search (the events are created once, on the first timed
+ *   call); 0 = off (default).  Read them with ivfpq_last_stage_ms. */
+#define IVFPQ_OPT_TIMING 2
 int ivfpq_index_set_option(ivfpq_index_t* index, int32_t option, int64_t value);
+
+/* Waits for the most recent timed search on this handle to finish and writes the device time
+ * in milliseconds of its filtering stage to ms[0] and of its LUT+scan+merge stage to ms[1].
+ * Returns IVFPQ_ERR_INVALID_ARGUMENT when timing is off or no search has run. */
+int ivfpq_last_stage_ms(const ivfpq_index_t* index, float* ms);
 
 /* Number of kernel launches the most recent search call on this handle enqueued. */
 int64_t ivfpq_last_launch_count(const ivfpq_index_t* index);

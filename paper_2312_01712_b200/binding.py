@@ -25,12 +25,13 @@ IVFPQ_ERR_WORKSPACE = -3
 IVFPQ_ERR_CUDA = -4
 IVFPQ_ERR_DEVICE_FLAG = -5
 IVFPQ_OPT_NSPLIT = 1
+IVFPQ_OPT_TIMING = 2
 
 EXPORTS = (
     "ivfpq_index_derived_bytes", "ivfpq_index_load", "ivfpq_index_free",
     "ivfpq_search_workspace_bytes", "ivfpq_search_dense", "ivfpq_search_sparse",
     "ivfpq_search_host_workspace_bytes", "ivfpq_search_host", "ivfpq_sync_status",
-    "ivfpq_index_set_option", "ivfpq_last_launch_count", "ivfpq_error_string",
+    "ivfpq_index_set_option", "ivfpq_last_launch_count", "ivfpq_last_stage_ms", "ivfpq_error_string",
     "ivfpq_debug_probes", "ivfpq_debug_search",
 )
 
@@ -89,6 +90,8 @@ def load_library() -> ctypes.CDLL:
     lib.ivfpq_index_set_option.restype = ctypes.c_int
     lib.ivfpq_last_launch_count.argtypes = [vp]
     lib.ivfpq_last_launch_count.restype = i64
+    lib.ivfpq_last_stage_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.ivfpq_last_stage_ms.restype = ctypes.c_int
     lib.ivfpq_error_string.argtypes = [ctypes.c_int]
     lib.ivfpq_error_string.restype = ctypes.c_char_p
     lib.ivfpq_debug_probes.argtypes = [vp, vp, i64, i32, vp, vp, vp, sz, vp]
@@ -181,6 +184,13 @@ def ivfpq_index_set_option(ix: IndexHandle, option: int, value: int) -> None:
 
 def ivfpq_last_launch_count(ix: IndexHandle) -> int:
     return int(load_library().ivfpq_last_launch_count(ix.handle))
+
+
+def ivfpq_last_stage_ms(ix: IndexHandle) -> Tuple[float, float]:
+    """(filtering ms, LUT+scan+merge ms) of the last search timed with IVFPQ_OPT_TIMING."""
+    ms = (ctypes.c_float * 2)()
+    _check(load_library().ivfpq_last_stage_ms(ix.handle, ms), "ivfpq_last_stage_ms")
+    return float(ms[0]), float(ms[1])
 
 
 def ivfpq_search_workspace_bytes(ix: IndexHandle, nq: int, nprobe: int, k: int) -> int:

@@ -76,12 +76,20 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
     int64_t launches = 0;
+    const bool timed = ix->timing != 0;
+    if (timed && !ix->ev_ready) {
+        for (int i = 0; i < 3; ++i)
+            if (cudaEventCreate(&ix->ev[i]) != cudaSuccess) return IVFPQ_ERR_CUDA;
+        ix->ev_ready = true;
+    }
     if (cudaMemsetAsync(ws + wl.status_off, 0, 16, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    if (timed && cudaEventRecord(ix->ev[0], st) != cudaSuccess) return IVFPQ_ERR_CUDA;
     int32_t* probe_ids = reinterpret_cast<int32_t*>(ws + wl.probe_ids_off);
     float* probe_d = reinterpret_cast<float*>(ws + wl.probe_d_off);
     if (launch_coarse(ix, a.queries, a.nq, a.nprobe, reinterpret_cast<float*>(ws + wl.coarse_off), wl.qchunk,
                       probe_ids, probe_d, reinterpret_cast<int*>(ws + wl.status_off), st, &launches) != cudaSuccess)
         return IVFPQ_ERR_CUDA;
+    if (timed && cudaEventRecord(ix->ev[1], st) != cudaSuccess) return IVFPQ_ERR_CUDA;
     const size_t pbytes = (size_t)a.nq * a.nprobe * 4;
     if (a.probe_ids_out &&
         cudaMemcpyAsync(a.probe_ids_out, probe_ids, pbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
@@ -90,6 +98,10 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
         return IVFPQ_ERR_CUDA;
     if (!probes_only) {
         if (launch_scan(a, wl, ws, st, &launches) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    }
+    if (timed) {
+        if (cudaEventRecord(ix->ev[2], st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+        ix->ev_recorded = true;
     }
     ix->last_launches = launches;
     return IVFPQ_OK;
@@ -184,6 +196,9 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->sm_count = sms;
     ix->nsplit_opt = 0;
     ix->last_launches = 0;
+    ix->timing = 0;
+    ix->ev_ready = false;
+    ix->ev_recorded = false;
 
     // list tables: built on the host, copied synchronously (pageable source)
     const size_t n1 = (size_t)desc->nlist + 1;
@@ -214,6 +229,8 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
 
 int ivfpq_index_free(ivfpq_index_t* index) {
     if (!index) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (index->ev_ready)
+        for (int i = 0; i < 3; ++i) cudaEventDestroy(index->ev[i]);
     delete index;
     return IVFPQ_OK;
 }
@@ -326,9 +343,21 @@ int ivfpq_index_set_option(ivfpq_index_t* index, int32_t option, int64_t value) 
             if (value < 0 || value > 64) return IVFPQ_ERR_INVALID_ARGUMENT;
             index->nsplit_opt = (int32_t)value;
             return IVFPQ_OK;
+        case IVFPQ_OPT_TIMING:
+            if (value != 0 && value != 1) return IVFPQ_ERR_INVALID_ARGUMENT;
+            index->timing = (int32_t)value;
+            return IVFPQ_OK;
         default:
             return IVFPQ_ERR_INVALID_ARGUMENT;
     }
+}
+
+int ivfpq_last_stage_ms(const ivfpq_index_t* index, float* ms) {
+    if (!index || !ms || !index->ev_ready || !index->ev_recorded) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (cudaEventSynchronize(index->ev[2]) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms[0], index->ev[0], index->ev[1]) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms[1], index->ev[1], index->ev[2]) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    return IVFPQ_OK;
 }
 
 int64_t ivfpq_last_launch_count(const ivfpq_index_t* index) { return index ? index->last_launches : 0; }

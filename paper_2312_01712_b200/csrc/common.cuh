@@ -40,6 +40,9 @@ struct ivfpq_index {
     int32_t sm_count;
     int32_t nsplit_opt;       // 0 = automatic
     mutable int64_t last_launches;
+    int32_t timing;           // IVFPQ_OPT_TIMING
+    mutable cudaEvent_t ev[3];  // start, after filtering, end (created lazily)
+    mutable bool ev_ready, ev_recorded;
 };
 
 namespace ivfpq {
