@@ -13,9 +13,10 @@ namespace {
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 struct DerivedLayout {
-    size_t list_off_off, list_blk_off, codes_off, total;
+    size_t list_off_off, list_blk_off, codes_off, cbt_off, total;
     int64_t nblocks, max_len;
     int32_t nw, vec16;
+    int32_t rot, gw[3], block_bytes;
 };
 
 // Validates the description and lays out the derived buffer.  Returns an IVFPQ_* code.
@@ -46,7 +47,11 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     out->list_blk_off = off;
     off = align_up(off + sizeof(int64_t) * (size_t)(d->nlist + 1), 256);
     out->codes_off = off;
-    off = align_up(off + (size_t)nblocks * kPointsPerBlock * out->nw * 4, 256);
+    out->rot = (rot_supported(d->nsub, d->dsub) && rot_group_widths(d->nsub, out->gw)) ? 1 : 0;
+    out->block_bytes = out->rot ? rot_block_bytes(out->gw) : kPointsPerBlock * out->nw * 4;
+    off = align_up(off + (size_t)nblocks * out->block_bytes, 256);
+    out->cbt_off = off;
+    if (out->rot) off = align_up(off + (size_t)d->nsub * 256 * d->dsub * 4, 256);
     out->total = off > 0 ? off : 256;
     return IVFPQ_OK;
 }
@@ -191,6 +196,10 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->nw = dl.nw;
     ix->vec16 = dl.vec16;
     ix->nblocks = dl.nblocks;
+    ix->rot = dl.rot;
+    for (int i = 0; i < 3; ++i) ix->gw[i] = dl.rot ? dl.gw[i] : 0;
+    ix->block_bytes = dl.block_bytes;
+    ix->cbt = reinterpret_cast<const float*>(base + dl.cbt_off);
     ix->max_list_len = dl.max_len;
     ix->device = dev;
     ix->sm_count = sms;
@@ -218,7 +227,8 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);  // the host arrays may go away after return
     delete[] blk;
     if (e == cudaSuccess)
-        e = launch_relayout(ix, desc->codes, reinterpret_cast<uint32_t*>(base + dl.codes_off), st);
+        e = launch_relayout(ix, desc->codes, reinterpret_cast<uint32_t*>(base + dl.codes_off),
+                            reinterpret_cast<float*>(base + dl.cbt_off), st);
     if (e != cudaSuccess) {
         delete ix;
         return IVFPQ_ERR_CUDA;

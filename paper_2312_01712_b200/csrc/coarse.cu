@@ -82,7 +82,8 @@ __global__ void __launch_bounds__(256) select_probes_kernel(const float* __restr
     __shared__ unsigned long long buf[kTopkCap];
     __shared__ int cnt;
     __shared__ unsigned long long tau;
-    TopkState t{buf, &cnt, &tau};
+    __shared__ int hist[kTopkHistInts];
+    TopkState t{buf, &cnt, &tau, hist};
     topk_init(t);
     const float* row = dist + (int64_t)blockIdx.x * nlist;
     for (int base = 0; base < nlist; base += blockDim.x) {
@@ -93,9 +94,9 @@ __global__ void __launch_bounds__(256) select_probes_kernel(const float* __restr
                 if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
             }
         }
-        topk_round_end(t, nprobe, blockDim.x);
+        topk_round_end<256>(t, nprobe, 256);
     }
-    topk_finalize(t, nprobe);
+    topk_finalize<256>(t, nprobe);
     const int64_t q = q0 + blockIdx.x;
     for (int i = threadIdx.x; i < nprobe; i += blockDim.x) {
         unsigned long long key = i < cnt ? buf[i] : kKeyPad;

@@ -34,6 +34,12 @@ struct ivfpq_index {
     int32_t nw;               // 4-byte code words per point (nsub rounded up to a multiple of 4)
     int32_t vec16;            // 1: words grouped by four (16-byte lane loads), 0: single words
     int64_t nblocks;          // total 32-point blocks
+    // rotated layout (scan_rot.cu): subspace groups of power-of-two width, codes stored per lane in
+    // the lane's own visiting order, codebook copied entry-major per group
+    int32_t rot;              // 1: rotated layout in use
+    int32_t gw[3];            // group widths, largest first, 0 = unused
+    int32_t block_bytes;      // bytes of one 32-point code block in the rotated layout
+    const float* cbt;         // [group][entry 0..255][column][dsub]
     int64_t max_list_len;
     // host state
     int32_t device;
@@ -87,7 +93,11 @@ struct WorkspaceLayout {
 WorkspaceLayout plan_workspace(const ivfpq_index* ix, int64_t nq, int32_t nprobe, int32_t k);
 
 // Launchers (return cudaError_t of the launch; count launches into *launches).
-cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_t* codes_il, cudaStream_t st);
+cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_t* codes_il, float* cbt,
+                            cudaStream_t st);
+bool rot_group_widths(int nsub, int w[3]);
+int rot_block_bytes(const int w[3]);
+bool rot_supported(int nsub, int dsub);
 cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,
                           float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
                           int* status, cudaStream_t st, int64_t* launches);

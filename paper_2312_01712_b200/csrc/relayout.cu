@@ -50,12 +50,84 @@ __global__ void __launch_bounds__(256) relayout_kernel(const uint8_t* __restrict
     }
 }
 
+__host__ __device__ inline int rot_lane_bytes(int w) { return w >= 16 ? w : (w == 8 ? 8 : (w > 0 ? 4 : 0)); }
+
+// Rotated layout (see scan_rot.cu): a 32-point block is a sequence of per-group chunks; in the
+// chunk of a group of width w the lane at position `lane` stores, as byte i (i < w), the code of
+// subspace s0 + ((lane ^ i) & (w-1)).  Lanes are interleaved at the granularity of the vector the
+// scan loads: 16 bytes (w >= 16), 8 bytes (w == 8) or 4 bytes (w <= 4).
+__global__ void __launch_bounds__(256) relayout_rot_kernel(const uint8_t* __restrict__ codes,
+                                                           const int64_t* __restrict__ list_off,
+                                                           const int64_t* __restrict__ list_blk, int nsub,
+                                                           int w0, int w1, int w2, int block_bytes,
+                                                           unsigned char* __restrict__ dst) {
+    const int list = blockIdx.x;
+    const int64_t p0 = list_off[list];
+    const int64_t len = list_off[list + 1] - p0;
+    const int64_t b0 = list_blk[list];
+    const int64_t nblk = list_blk[list + 1] - b0;
+    const int gw[3] = {w0, w1, w2};
+    for (int64_t i = threadIdx.x; i < nblk * kPointsPerBlock; i += blockDim.x) {
+        const int lane = (int)(i & 31);
+        const int64_t b = i >> 5;
+        const int64_t pos = i;
+        const uint8_t* src = codes + (p0 + pos) * nsub;
+        unsigned char* blk = dst + (b0 + b) * block_bytes;
+        int s0 = 0, chunk = 0;
+        for (int g = 0; g < 3; ++g) {
+            const int w = gw[g];
+            if (w == 0) break;
+            const int lb = rot_lane_bytes(w);
+            const int vec = lb >= 16 ? 16 : lb;  // bytes per lane per vector
+            for (int i2 = 0; i2 < lb; ++i2) {
+                unsigned char v = 0;
+                if (i2 < w && pos < len) v = src[s0 + ((lane ^ i2) & (w - 1))];
+                // vector number i2 / vec, lanes interleaved per vector
+                blk[chunk + (i2 / vec) * 32 * vec + lane * vec + (i2 % vec)] = v;
+            }
+            s0 += w;
+            chunk += 32 * lb;
+        }
+    }
+}
+
+// Entry-major codebook copy per group: cbt[s0*256*dsub + ((e*w + c)*dsub + j)] = cb[s0+c][e][j];
+// entries e >= ksub are zero.
+__global__ void __launch_bounds__(256) relayout_cbt_kernel(const float* __restrict__ cb, int nsub, int dsub,
+                                                           int ksub, int w0, int w1, int w2,
+                                                           float* __restrict__ cbt) {
+    const int gw[3] = {w0, w1, w2};
+    const int total = nsub * 256 * dsub;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        int s0 = 0, g = 0;
+        while (g < 2 && i >= (s0 + gw[g]) * 256 * dsub) {
+            s0 += gw[g];
+            ++g;
+        }
+        const int w = gw[g];
+        const int r = i - s0 * 256 * dsub;
+        const int j = r % dsub;
+        const int c = (r / dsub) % w;
+        const int e = r / (dsub * w);
+        cbt[i] = e < ksub ? cb[((size_t)(s0 + c) * ksub + e) * dsub + j] : 0.0f;
+    }
+}
+
 }  // namespace
 
-cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_t* codes_il, cudaStream_t st) {
-    if (ix->nlist > 0 && ix->nblocks > 0)
+cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_t* codes_il, float* cbt,
+                            cudaStream_t st) {
+    if (ix->rot) {
+        if (ix->nblocks > 0)
+            relayout_rot_kernel<<<ix->nlist, 256, 0, st>>>(codes, ix->list_off, ix->list_blk, ix->nsub, ix->gw[0],
+                                                           ix->gw[1], ix->gw[2], ix->block_bytes,
+                                                           reinterpret_cast<unsigned char*>(codes_il));
+        relayout_cbt_kernel<<<64, 256, 0, st>>>(ix->cb, ix->nsub, ix->dsub, ix->ksub, ix->gw[0], ix->gw[1],
+                                                ix->gw[2], cbt);
+    } else if (ix->nlist > 0 && ix->nblocks > 0) {
         relayout_kernel<<<ix->nlist, 256, 0, st>>>(codes, ix->list_off, ix->list_blk, ix->nsub, ix->nw,
                                                    ix->vec16, codes_il);
+    }
     return cudaGetLastError();
 }
 

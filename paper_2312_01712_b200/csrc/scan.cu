@@ -14,6 +14,7 @@
 //   4. feeds (distance, id) into a CTA-wide streaming top-k.
 // The table is never written to global memory.
 #include "common.cuh"
+#include "scan_common.cuh"
 #include "topk.cuh"
 
 namespace ivfpq {
@@ -24,43 +25,12 @@ constexpr int kBlocksPerWarpRound = 4;                                          
 constexpr int kRoundPoints = kScanThreads * kBlocksPerWarpRound;                  // candidates per round, CTA-wide
 static_assert(IVFPQ_MAX_K + kRoundPoints <= kTopkCap, "candidate buffer too small for a round");
 
-struct ScanParams {
-    const float* cent;
-    const float* cb;
-    const int32_t* ids;
-    const uint32_t* codes_il;
-    const int64_t* list_off;
-    const int64_t* list_blk;
-    int d, nlist, nsub, dsub, ksub, nw;
-    const float* queries;
-    const int32_t* probe_ids;
-    int nprobe;
-    const float* radius;
-    int radius_mode;
-    float scale;
-    float miss_penalty;
-    int dense;
-    int k;
-    int nsplit;
-    float* out_dist;
-    int32_t* out_ids;
-    unsigned long long* partial;
-    int* status;
-    // stage dumps (DBG instantiations only)
-    uint32_t* masks;
-    int64_t* visit_count;
-    int64_t visit_stride;
-    unsigned long long* visit_hits;
-    float* visit_dist;
-    int32_t* visit_ids;
-};
-
 __host__ __device__ inline size_t scan_smem_bytes(int nw, int d, int nprobe, bool dbg) {
     size_t b = (size_t)kTopkCap * 8;              // candidate keys
     b += (size_t)nw * 4 * 256 * 4;                // table, padded subspaces included
     b += align_up((size_t)d * 4, 16);             // residual
     b += IVFPQ_MAX_NSUB * 4;                      // squared thresholds
-    b += 32;                                      // counters
+    b += 32 + kTopkHistInts * 4;                  // counters, selection histogram
     if (dbg) b += IVFPQ_MAX_NSUB * 8 * 4 + (size_t)(nprobe + 1) * 8;
     return b;
 }
@@ -97,12 +67,13 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(const ScanParams p) 
     float* r2 = res + align_up((size_t)d * 4, 16) / 4;
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + IVFPQ_MAX_NSUB);
     int* cnt_p = reinterpret_cast<int*>(tau_p + 1);
-    uint32_t* hitmask = reinterpret_cast<uint32_t*>(tau_p + 4);          // DBG only
+    int* hist_p = reinterpret_cast<int*>(tau_p + 4);
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(hist_p + kTopkHistInts);  // DBG only
     long long* vprefix = reinterpret_cast<long long*>(hitmask + IVFPQ_MAX_NSUB * 8);  // DBG only
 
     const int64_t q = blockIdx.x / p.nsplit;
     const int split = blockIdx.x % p.nsplit;
-    TopkState t{kbuf, cnt_p, tau_p};
+    TopkState t{kbuf, cnt_p, tau_p, hist_p};
 
     // squared thresholds of this query, one per subspace; the miss constant
     if (tid < nsub) {
@@ -254,11 +225,11 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(const ScanParams p) 
                     }
                 }
             }
-            topk_round_end(t, p.k, kRoundPoints);
+            topk_round_end<kScanThreads>(t, p.k, kRoundPoints);
         }
     }
 
-    topk_finalize(t, p.k);
+    topk_finalize<kScanThreads>(t, p.k);
     const int n = *cnt_p;
     if (p.nsplit == 1) {
         for (int i = tid; i < p.k; i += kScanThreads) {
@@ -280,7 +251,8 @@ __global__ void __launch_bounds__(kScanThreads) merge_kernel(const unsigned long
     __shared__ unsigned long long buf[kTopkCap];
     __shared__ int cnt;
     __shared__ unsigned long long tau;
-    TopkState t{buf, &cnt, &tau};
+    __shared__ int hist[kTopkHistInts];
+    TopkState t{buf, &cnt, &tau, hist};
     topk_init(t);
     const int64_t q = blockIdx.x;
     const unsigned long long* src = partial + q * nsplit * (int64_t)k;
@@ -293,9 +265,9 @@ __global__ void __launch_bounds__(kScanThreads) merge_kernel(const unsigned long
                 if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
             }
         }
-        topk_round_end(t, k, kScanThreads);
+        topk_round_end<kScanThreads>(t, k, kScanThreads);
     }
-    topk_finalize(t, k);
+    topk_finalize<kScanThreads>(t, k);
     for (int i = threadIdx.x; i < k; i += kScanThreads) {
         const unsigned long long key = i < cnt ? buf[i] : kKeyPad;
         out_dist[q * k + i] = __uint_as_float((uint32_t)(key >> 32));
@@ -329,6 +301,7 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     ScanParams sp{};
     sp.cent = ix->cent;
     sp.cb = ix->cb;
+    sp.cbt = ix->cbt;
     sp.ids = ix->ids;
     sp.codes_il = ix->codes_il;
     sp.list_off = ix->list_off;
@@ -362,7 +335,13 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
 
     const size_t smem = scan_smem_bytes(ix->nw, ix->d, a.nprobe, a.debug);
     const int64_t grid = a.nq * sp.nsplit;
-    cudaError_t e = a.debug ? dispatch<true>(ix, sp, grid, smem, st) : dispatch<false>(ix, sp, grid, smem, st);
+    cudaError_t e;
+    if (ix->rot && ix->nsub == 16 && ix->dsub == 8)
+        e = launch_scan_pers(ix, sp, grid, a.debug, a.nprobe, st);
+    else if (ix->rot)
+        e = launch_scan_rot(ix, sp, grid, a.debug, a.nprobe, st);
+    else
+        e = a.debug ? dispatch<true>(ix, sp, grid, smem, st) : dispatch<false>(ix, sp, grid, smem, st);
     if (e != cudaSuccess) return e;
     *launches += 1;
     if (sp.nsplit > 1) {

@@ -1,0 +1,50 @@
+// Parameters shared by the list-scan kernels.
+#pragma once
+
+#include "common.cuh"
+
+namespace ivfpq {
+
+struct ScanParams {
+    const float* cent;
+    const float* cb;
+    const float* cbt;
+    const int32_t* ids;
+    const uint32_t* codes_il;
+    const int64_t* list_off;
+    const int64_t* list_blk;
+    int d, nlist, nsub, dsub, ksub, nw;
+    const float* queries;
+    const int32_t* probe_ids;
+    int nprobe;
+    const float* radius;
+    int radius_mode;
+    float scale;
+    float miss_penalty;
+    int dense;
+    int k;
+    int nsplit;
+    float* out_dist;
+    int32_t* out_ids;
+    unsigned long long* partial;
+    int* status;
+    // stage dumps (DBG instantiations only)
+    uint32_t* masks;
+    int64_t* visit_count;
+    int64_t visit_stride;
+    unsigned long long* visit_hits;
+    float* visit_dist;
+    int32_t* visit_ids;
+};
+
+
+// Rotated-layout scan (scan_rot.cu); returns cudaErrorNotSupported when the index shape has no
+// specialised instance.
+cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, bool debug,
+                            int nprobe, cudaStream_t st);
+
+// Persistent register-resident-codebook scan for the 16 x 8 quantizer (scan_pers.cu).
+cudaError_t launch_scan_pers(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
+                             cudaStream_t st);
+
+}  // namespace ivfpq

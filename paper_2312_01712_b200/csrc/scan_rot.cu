@@ -1,0 +1,351 @@
+// Rotated-layout variant of the fused selective-LUT / list-scan / top-k kernel.
+//
+// Same computation as scan.cu (paper Sec. 2.1 steps B-D with the selection of Sec. 3.1 /
+// Algorithm 2 and the miss constant of Sec. 4.3), different shared-memory organisation, chosen
+// so that the table gathers of a warp never collide on a bank whatever the codes are:
+//
+//   * the subspaces are split into groups of width w (a power of two, 32 or less); a group's table
+//     is stored entry-major, LUT_g[entry][32 columns], and column (copy*w + c) of every row holds
+//     the value of subspace s0+c, replicated 32/w times;
+//   * a lane (one point per lane) walks its w code bytes of the group in a lane-specific order:
+//     at step i it looks up subspace s0 + ((lane ^ i) & (w-1)) in column lane ^ i.  At any step
+//     the 32 lanes therefore touch the 32 different columns = 32 different banks;
+//   * the code bytes are stored in that rotated order when the index is loaded, so byte i of the
+//     lane's vector is the one it needs at step i.
+// The table is built with lanes running over the columns of a row (not over entries), reading
+// the codebook from an entry-major copy made at load time, so both the codebook loads and the
+// table stores are contiguous / conflict-free.
+#include "common.cuh"
+#include "scan_common.cuh"
+#include "topk.cuh"
+
+namespace ivfpq {
+
+namespace {
+
+constexpr int kLutGroupFloats = 256 * 32;  // one group table: 256 entries x 32 columns
+
+__host__ __device__ constexpr int lane_bytes(int w) { return w >= 16 ? w : (w == 8 ? 8 : (w > 0 ? 4 : 0)); }
+
+template <int W0, int W1, int W2>
+struct Groups {
+    static constexpr int kNum = (W0 > 0) + (W1 > 0) + (W2 > 0);
+    static constexpr int kNsub = W0 + W1 + W2;
+    static constexpr int kBlockBytes = 32 * (lane_bytes(W0) + lane_bytes(W1) + lane_bytes(W2));
+    __host__ __device__ static constexpr int width(int g) { return g == 0 ? W0 : (g == 1 ? W1 : W2); }
+    __host__ __device__ static constexpr int s0(int g) { return g == 0 ? 0 : (g == 1 ? W0 : W0 + W1); }
+    // byte offset of group g's chunk inside a 32-point block
+    __host__ __device__ static constexpr int chunk_off(int g) {
+        return 32 * (g == 0 ? 0 : (g == 1 ? lane_bytes(W0) : lane_bytes(W0) + lane_bytes(W1)));
+    }
+};
+
+__host__ __device__ inline size_t rot_smem_bytes(int ngroups, int d, int nprobe, bool dbg) {
+    size_t b = (size_t)kTopkCap * 8;
+    b += (size_t)ngroups * kLutGroupFloats * 4;
+    b += align_up((size_t)d * 4, 16);
+    b += IVFPQ_MAX_NSUB * 4;
+    b += 32 + kTopkHistInts * 4;
+    if (dbg) b += IVFPQ_MAX_NSUB * 8 * 4 + (size_t)(nprobe + 1) * 8;
+    return b;
+}
+
+// Table of one group for one (query, cluster): thread t owns column c = t & (W-1) and the
+// entries u, u + NT/W, ... with u = t / W.
+template <int W, int DSUB, int NT, bool DBG>
+__device__ __forceinline__ void build_group(float* __restrict__ lutg, const float* __restrict__ cbt_g,
+                                            const float* __restrict__ res_g, const float* __restrict__ r2_g,
+                                            int ksub, bool dense, float P, uint32_t* hitmask_g) {
+    constexpr int EP = NT / W;      // entries per pass
+    constexpr int NCOPY = 32 / W;
+    const int t = threadIdx.x;
+    const int c = t & (W - 1);
+    const int u = t / W;
+    const int usub = (t & 31) / W;  // which of the warp's entries this lane works on
+    float r[DSUB];
+#pragma unroll
+    for (int j = 0; j < DSUB; ++j) r[j] = res_g[c * DSUB + j];
+    const float thr = r2_g[c];
+#pragma unroll 2
+    for (int e = u; e < 256; e += EP) {
+        float d2 = 0.0f;
+        bool hit = false;
+        if (e < ksub) {
+            const float* ent = cbt_g + ((size_t)e * W + c) * DSUB;
+            if constexpr (DSUB % 4 == 0) {
+#pragma unroll
+                for (int j4 = 0; j4 < DSUB / 4; ++j4) {
+                    const float4 ev = __ldg(reinterpret_cast<const float4*>(ent) + j4);
+                    float tt;
+                    tt = __fsub_rn(r[4 * j4 + 0], ev.x); d2 = __fmaf_rn(tt, tt, d2);
+                    tt = __fsub_rn(r[4 * j4 + 1], ev.y); d2 = __fmaf_rn(tt, tt, d2);
+                    tt = __fsub_rn(r[4 * j4 + 2], ev.z); d2 = __fmaf_rn(tt, tt, d2);
+                    tt = __fsub_rn(r[4 * j4 + 3], ev.w); d2 = __fmaf_rn(tt, tt, d2);
+                }
+            } else if constexpr (DSUB % 2 == 0) {
+#pragma unroll
+                for (int j2 = 0; j2 < DSUB / 2; ++j2) {
+                    const float2 ev = __ldg(reinterpret_cast<const float2*>(ent) + j2);
+                    float tt;
+                    tt = __fsub_rn(r[2 * j2 + 0], ev.x); d2 = __fmaf_rn(tt, tt, d2);
+                    tt = __fsub_rn(r[2 * j2 + 1], ev.y); d2 = __fmaf_rn(tt, tt, d2);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < DSUB; ++j) {
+                    float tt = __fsub_rn(r[j], __ldg(ent + j));
+                    d2 = __fmaf_rn(tt, tt, d2);
+                }
+            }
+            hit = dense || d2 <= thr;
+        }
+        const float val = hit ? d2 : P;
+        float* row = lutg + e * 32 + c;
+#pragma unroll
+        for (int it = 0; it < NCOPY; ++it) {
+            const int copy = (it + usub) & (NCOPY - 1);  // lanes of a warp write different columns
+            row[copy * W] = val;
+        }
+        if (DBG && hit) atomicOr(&hitmask_g[c * 8 + (e >> 5)], 1u << (e & 31));
+    }
+}
+
+// Sum of the table values of one group for the lane's point.  `bytes` holds the lane's code bytes
+// of the group in rotated order.
+template <int W, bool DBG>
+__device__ __forceinline__ void gather_group(const float* __restrict__ lutg, const uint32_t* words, int lane,
+                                             int s0, const uint32_t* hitmask, float& acc,
+                                             unsigned long long& hs) {
+#pragma unroll
+    for (int i = 0; i < W; ++i) {
+        const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 0xFFu;
+        acc += lutg[code * 32 + (lane ^ i)];
+        if (DBG) {
+            const int s = s0 + ((lane ^ i) & (W - 1));
+            hs |= (unsigned long long)((hitmask[s * 8 + (code >> 5)] >> (code & 31)) & 1u) << s;
+        }
+    }
+}
+
+template <int W>
+__device__ __forceinline__ void load_group_codes(const unsigned char* __restrict__ chunk, int lane,
+                                                 uint32_t* words) {
+    if constexpr (W >= 16) {
+#pragma unroll
+        for (int v = 0; v < W / 16; ++v) {
+            const uint4 x = __ldg(reinterpret_cast<const uint4*>(chunk) + v * 32 + lane);
+            words[4 * v + 0] = x.x;
+            words[4 * v + 1] = x.y;
+            words[4 * v + 2] = x.z;
+            words[4 * v + 3] = x.w;
+        }
+    } else if constexpr (W == 8) {
+        const uint2 x = __ldg(reinterpret_cast<const uint2*>(chunk) + lane);
+        words[0] = x.x;
+        words[1] = x.y;
+    } else {
+        words[0] = __ldg(reinterpret_cast<const uint32_t*>(chunk) + lane);
+    }
+}
+
+template <int W0, int W1, int W2, int DSUB, int NT, bool DBG>
+__global__ void __launch_bounds__(NT) scan_rot_kernel(const ScanParams p) {
+    using GR = Groups<W0, W1, W2>;
+    constexpr int kWarps = NT / 32;
+    constexpr int kBlocksPerWarpRound = 1024 / NT;       // 1024 candidates per round, CTA-wide
+    static_assert(IVFPQ_MAX_K + 1024 <= kTopkCap, "candidate buffer too small for a round");
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int nsub = GR::kNsub;
+    const int ksub = p.ksub;
+    const int d = p.d;
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+
+    unsigned long long* kbuf = reinterpret_cast<unsigned long long*>(smem);
+    float* lut = reinterpret_cast<float*>(smem + (size_t)kTopkCap * 8);
+    float* res = lut + (size_t)GR::kNum * kLutGroupFloats;
+    float* r2 = res + align_up((size_t)d * 4, 16) / 4;
+    unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + IVFPQ_MAX_NSUB);
+    int* cnt_p = reinterpret_cast<int*>(tau_p + 1);
+    int* hist_p = reinterpret_cast<int*>(tau_p + 4);
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(hist_p + kTopkHistInts);           // DBG only
+    long long* vprefix = reinterpret_cast<long long*>(hitmask + IVFPQ_MAX_NSUB * 8);   // DBG only
+
+    const int64_t q = blockIdx.x / p.nsplit;
+    const int split = blockIdx.x % p.nsplit;
+    TopkState t{kbuf, cnt_p, tau_p, hist_p};
+
+    if (tid < nsub) {
+        float v = 0.0f;
+        if (!p.dense) {
+            const float* rad = p.radius_mode == 1 ? p.radius + q * nsub : p.radius;
+            float r = __fmul_rn(rad[tid], p.scale);
+            v = __fmul_rn(r, r);
+        }
+        r2[tid] = v;
+    }
+    if (DBG && tid == 0) {
+        long long run = 0;
+        for (int i = 0; i < p.nprobe; ++i) {
+            vprefix[i] = run;
+            int c = p.probe_ids[q * p.nprobe + i];
+            if (c >= 0 && c < p.nlist) run += p.list_off[c + 1] - p.list_off[c];
+        }
+        vprefix[p.nprobe] = run;
+        if (p.visit_count) p.visit_count[q] = run;
+    }
+    topk_init(t);
+    float P = 0.0f;
+    if (!p.dense) {
+        if (p.miss_penalty >= 0.0f) {
+            P = p.miss_penalty;
+        } else {
+            for (int s = 0; s < nsub; ++s) P = __fadd_rn(P, r2[s]);
+        }
+    }
+
+    for (int pi = split; pi < p.nprobe; pi += p.nsplit) {
+        const int c = p.probe_ids[q * p.nprobe + pi];
+        if (c < 0 || c >= p.nlist) {
+            if (tid == 0) atomicOr(p.status, kFlagBadList);
+            continue;
+        }
+        __syncthreads();  // the previous cluster's scan no longer reads the tables
+        for (int j = tid; j < d; j += NT) res[j] = __fsub_rn(p.queries[q * d + j], p.cent[(int64_t)c * d + j]);
+        if (DBG)
+            for (int i = tid; i < IVFPQ_MAX_NSUB * 8; i += NT) hitmask[i] = 0;
+        __syncthreads();
+
+        // ---- selective tables, one per group ----
+        build_group<W0, DSUB, NT, DBG>(lut, p.cbt, res, r2, ksub, p.dense, P, hitmask);
+        if constexpr (W1 > 0)
+            build_group<W1, DSUB, NT, DBG>(lut + kLutGroupFloats, p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
+                                           res + GR::s0(1) * DSUB, r2 + GR::s0(1), ksub, p.dense, P,
+                                           hitmask + GR::s0(1) * 8);
+        if constexpr (W2 > 0)
+            build_group<W2, DSUB, NT, DBG>(lut + 2 * kLutGroupFloats, p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
+                                           res + GR::s0(2) * DSUB, r2 + GR::s0(2), ksub, p.dense, P,
+                                           hitmask + GR::s0(2) * 8);
+        __syncthreads();
+        if (DBG && p.masks)
+            for (int i = tid; i < nsub * 8; i += NT) p.masks[(q * p.nprobe + pi) * nsub * 8 + i] = hitmask[i];
+
+        // ---- scan the cluster ----
+        const int64_t p0 = p.list_off[c];
+        const int64_t len = p.list_off[c + 1] - p0;
+        const int64_t b0 = p.list_blk[c];
+        const int64_t nblk = p.list_blk[c + 1] - b0;
+        if (nblk != (len + kPointsPerBlock - 1) / kPointsPerBlock || len < 0) {
+            if (tid == 0) atomicOr(p.status, kFlagBadList);
+            continue;
+        }
+        const unsigned char* cbase = reinterpret_cast<const unsigned char*>(p.codes_il) + b0 * GR::kBlockBytes;
+        for (int64_t bb = 0; bb < nblk; bb += kWarps * kBlocksPerWarpRound) {
+            const unsigned long long tau = *tau_p;
+            const uint32_t tau_hi = (uint32_t)(tau >> 32);
+#pragma unroll 1
+            for (int r = 0; r < kBlocksPerWarpRound; ++r) {
+                const int64_t blk = bb + r * kWarps + warp;
+                if (blk >= nblk) break;
+                const unsigned char* bp = cbase + blk * GR::kBlockBytes;
+                uint32_t w0[W0 >= 4 ? W0 / 4 : 1];
+                uint32_t w1[W1 >= 4 ? W1 / 4 : 1];
+                uint32_t w2[W2 >= 4 ? W2 / 4 : 1];
+                load_group_codes<W0>(bp, lane, w0);
+                if constexpr (W1 > 0) load_group_codes<W1>(bp + GR::chunk_off(1), lane, w1);
+                if constexpr (W2 > 0) load_group_codes<W2>(bp + GR::chunk_off(2), lane, w2);
+                float acc = 0.0f;
+                unsigned long long hs = 0;
+                gather_group<W0, DBG>(lut, w0, lane, 0, hitmask, acc, hs);
+                if constexpr (W1 > 0) gather_group<W1, DBG>(lut + kLutGroupFloats, w1, lane, GR::s0(1), hitmask, acc, hs);
+                if constexpr (W2 > 0)
+                    gather_group<W2, DBG>(lut + 2 * kLutGroupFloats, w2, lane, GR::s0(2), hitmask, acc, hs);
+                const int64_t pos = blk * kPointsPerBlock + lane;
+                if (pos < len) {
+                    if (DBG) {
+                        const int64_t vi = vprefix[pi] + pos;
+                        if (vi < p.visit_stride) {
+                            if (p.visit_hits) p.visit_hits[q * p.visit_stride + vi] = hs;
+                            if (p.visit_dist) p.visit_dist[q * p.visit_stride + vi] = acc;
+                            if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[p0 + pos];
+                        }
+                    }
+                    if (__float_as_uint(acc) <= tau_hi) {
+                        const unsigned long long key = make_key(acc, (uint32_t)p.ids[p0 + pos]);
+                        if (key < tau) {
+                            if (!topk_push(t, key)) atomicOr(p.status, kFlagOverflow);
+                        }
+                    }
+                }
+            }
+            topk_round_end<NT>(t, p.k, 1024);
+        }
+    }
+
+    topk_finalize<NT>(t, p.k);
+    const int n = *cnt_p;
+    if (p.nsplit == 1) {
+        for (int i = tid; i < p.k; i += NT) {
+            const unsigned long long key = i < n ? kbuf[i] : kKeyPad;
+            p.out_dist[q * p.k + i] = __uint_as_float((uint32_t)(key >> 32));
+            p.out_ids[q * p.k + i] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
+        }
+    } else {
+        unsigned long long* dst = p.partial + (q * p.nsplit + split) * p.k;
+        for (int i = tid; i < p.k; i += NT) dst[i] = i < n ? kbuf[i] : kKeyPad;
+    }
+}
+
+template <int W0, int W1, int W2, int DSUB, int NT>
+cudaError_t launch_rot(const ScanParams& sp, int64_t grid, bool debug, int nprobe, cudaStream_t st) {
+    const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kNum, sp.d, nprobe, debug);
+    cudaError_t e;
+    if (debug) {
+        auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, true>;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)grid, NT, smem, st>>>(sp);
+    } else {
+        auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, false>;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)grid, NT, smem, st>>>(sp);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// Decomposition of nsub into at most three power-of-two group widths (largest first), or false.
+bool rot_group_widths(int nsub, int w[3]) {
+    w[0] = w[1] = w[2] = 0;
+    int rest = nsub, n = 0;
+    for (int cand = 32; cand >= 1 && rest > 0; cand >>= 1) {
+        while (rest >= cand) {
+            if (n == 3) return false;
+            w[n++] = cand;
+            rest -= cand;
+        }
+    }
+    return rest == 0;
+}
+
+int rot_block_bytes(const int w[3]) { return 32 * (lane_bytes(w[0]) + lane_bytes(w[1]) + lane_bytes(w[2])); }
+
+bool rot_supported(int nsub, int dsub) {
+    return (nsub == 16 && dsub == 8) || (nsub == 48 && dsub == 2) || (nsub == 50 && dsub == 4) ||
+           (nsub == 8 && dsub == 4) || (nsub == 12 && dsub == 2);
+}
+
+cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, bool debug, int nprobe,
+                            cudaStream_t st) {
+    if (ix->nsub == 16 && ix->dsub == 8) return launch_rot<16, 0, 0, 8, 256>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 48 && ix->dsub == 2) return launch_rot<32, 16, 0, 2, 256>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 50 && ix->dsub == 4) return launch_rot<32, 16, 2, 4, 256>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 8 && ix->dsub == 4) return launch_rot<8, 0, 0, 4, 256>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 12 && ix->dsub == 2) return launch_rot<8, 4, 0, 2, 256>(sp, grid, debug, nprobe, st);
+    return cudaErrorNotSupported;
+}
+
+}  // namespace ivfpq
