@@ -83,6 +83,37 @@ def test_hand_worked_example_dense_and_sparse():
     assert sp4["masks"][0, 0, 0, 0] == 0b1111 and sp4["masks"][0, 0, 1, 0] == 0b1111
 
 
+def _golden(name):
+    import os
+    out = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
+        for line in f:
+            line = line.split("#")[0].strip()
+            if line:
+                key, rest = line.split(None, 1)
+                out[key] = rest
+    return out
+
+
+def test_golden_hand_example_file():
+    """The same hand-worked example read from tests/golden/hand_example.txt (values written by
+    hand, with the passages they follow), so the fixture and the in-line arithmetic cannot drift."""
+    g = _golden("hand_example.txt")
+    nums = lambda k: [float(x) for x in g[k].split()]
+    idx = hand_index()
+    assert idx.coarse_centroids.ravel().tolist() == [float(x) for x in g["centroids"].replace(";", " ").split()]
+    assert idx.codebooks[0].ravel().tolist() == nums("codebook0") and idx.codebooks[1].ravel().tolist() == nums("codebook1")
+    q = np.array([nums("query")], F32)
+    pid, pd = oracle.coarse(idx, q, 2)
+    assert pid[0].tolist() == nums("probes") and pd[0].tolist() == nums("probe_d")
+    o = oracle.search(idx, q, 2, 5, dense=True)
+    assert o["ids"][0].tolist() == nums("dense_ids") and o["dist"][0].tolist() == nums("dense_dist")
+    o = oracle.search(idx, q, 2, 5, radius=np.array(nums("radius"), F32), dumps=True, visit_stride=8)
+    assert o["ids"][0].tolist() == nums("sparse_ids") and o["dist"][0].tolist() == nums("sparse_dist")
+    assert [int(o["masks"][0, 0, s, 0]) for s in range(2)] == [int(x, 2) for x in g["masks_list0"].split()]
+    assert o["visit_hits"][0, :5].tolist() == [int(x, 2) for x in g["hitsets"].split()]
+
+
 # ---------------------------------------------------------------------------------------------
 # P1: radius -> infinity equals dense, bit for bit
 # ---------------------------------------------------------------------------------------------
