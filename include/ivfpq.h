@@ -45,6 +45,7 @@ extern "C" {
 #define IVFPQ_ERR_WORKSPACE (-3)        /* workspace or derived buffer too small / misaligned     */
 #define IVFPQ_ERR_CUDA (-4)             /* a CUDA runtime call or kernel launch failed            */
 #define IVFPQ_ERR_DEVICE_FLAG (-5)      /* a kernel raised its bounds / bounded-wait error flag   */
+#define IVFPQ_ERR_STATIC_LIMIT (-6)     /* index too large for the scratch built into the library */
 
 #define IVFPQ_MAX_K 1024
 #define IVFPQ_MAX_NPROBE 1024
@@ -144,6 +145,35 @@ int ivfpq_last_stage_ms(const ivfpq_index_t* index, float* ms);
 
 /* Number of kernel launches the most recent search call on this handle enqueued. */
 int64_t ivfpq_last_launch_count(const ivfpq_index_t* index);
+
+/* Filtering stage for callers that cannot provide or allocate device scratch.  (The paper has no
+ * counterpart: this is the same computation as the filtering step of ivfpq_search_*, packaged for a
+ * deployment constraint.)
+ *
+ * Who needs it: code that runs where device allocation is off the table - a serving loop that
+ * handed all free device memory to its own pool at start-up, a plug-in that may not call
+ * cudaMalloc because the host application forbids the implicit device-wide synchronisation it
+ * causes, a caller that has no allocator to ask for a workspace buffer at all.  Such callers still
+ * own their inputs and outputs; what they lack is a place for the [queries][nlist] distance tile
+ * between the distance kernel and the selection kernel.  Here that tile lives in a fixed array of
+ * IVFPQ_STATIC_SCRATCH_BYTES inside the library image: every GPU on which the library is loaded
+ * holds those bytes until the process exits.
+ *
+ * Same results as ivfpq_debug_probes: probe_ids dev [nq][nprobe] ascending by (distance, cluster
+ * id), probe_d dev [nq][nprobe].  The query batch is processed in chunks that fit the array.
+ * The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine) and is
+ * asynchronous on `stream`.  The current device must be the one the index was loaded on.
+ *   - indexes with nlist > IVFPQ_STATIC_MAX_NLIST are rejected with IVFPQ_ERR_STATIC_LIMIT;
+ *   - the first call on a device looks up the device address of the array (one runtime query,
+ *     cached per device); make that first call outside any stream capture;
+ *   - all calls on a device share the one array, which keeps whatever the previous call left in
+ *     it; the call clears the status word it needs zeroed and overwrites the rest before reading
+ *     it, but two calls whose kernels overlap on the GPU (different streams, different host
+ *     threads) race on it: serialise them. */
+#define IVFPQ_STATIC_SCRATCH_BYTES (8u << 20)
+#define IVFPQ_STATIC_MAX_NLIST 16384
+int ivfpq_probe_static(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                       int32_t* probe_ids, float* probe_d, void* stream);
 
 const char* ivfpq_error_string(int code);
 

@@ -24,6 +24,9 @@ IVFPQ_ERR_UNSUPPORTED = -2
 IVFPQ_ERR_WORKSPACE = -3
 IVFPQ_ERR_CUDA = -4
 IVFPQ_ERR_DEVICE_FLAG = -5
+IVFPQ_ERR_STATIC_LIMIT = -6
+IVFPQ_STATIC_SCRATCH_BYTES = 8 << 20
+IVFPQ_STATIC_MAX_NLIST = 16384
 IVFPQ_OPT_NSPLIT = 1
 IVFPQ_OPT_TIMING = 2
 
@@ -32,7 +35,7 @@ EXPORTS = (
     "ivfpq_search_workspace_bytes", "ivfpq_search_dense", "ivfpq_search_sparse",
     "ivfpq_search_host_workspace_bytes", "ivfpq_search_host", "ivfpq_sync_status",
     "ivfpq_index_set_option", "ivfpq_last_launch_count", "ivfpq_last_stage_ms", "ivfpq_error_string",
-    "ivfpq_debug_probes", "ivfpq_debug_search",
+    "ivfpq_debug_probes", "ivfpq_debug_search", "ivfpq_probe_static",
 )
 
 
@@ -99,6 +102,8 @@ def load_library() -> ctypes.CDLL:
     lib.ivfpq_debug_search.argtypes = [vp, vp, i64, i32, ctypes.POINTER(ivfpq_radius_t), i32, vp, vp,
                                        vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
     lib.ivfpq_debug_search.restype = ctypes.c_int
+    lib.ivfpq_probe_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+    lib.ivfpq_probe_static.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -314,3 +319,24 @@ def ivfpq_debug_search(ix: IndexHandle, queries: torch.Tensor, nprobe: int, k: i
     if visit_stride > 0:
         res.update(visit_hits=vh, visit_dist=vd, visit_ids=vi)
     return res
+
+
+def ivfpq_probe_static(ix: IndexHandle, queries: torch.Tensor, nprobe: int,
+                       out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None):
+    """Filtering stage through the entry point that needs no workspace: the distance tile lives
+    in an array built into the library (see `ivfpq_probe_static` in ivfpq.h for who needs this
+    and for its limits).  Pass `out=(probe_ids, probe_d)` to keep even the outputs out of the
+    allocator; otherwise they are new torch tensors.  Returns (probe_ids [nq, nprobe] int32,
+    probe_d [nq, nprobe] fp32)."""
+    if queries.dtype != torch.float32 or not queries.is_cuda or not queries.is_contiguous() or queries.dim() != 2 \
+            or queries.shape[1] != ix.d:
+        raise ValueError("queries must be a contiguous fp32 CUDA tensor [nq, d]")
+    nq = queries.shape[0]
+    if out is None:
+        pid = torch.empty((nq, nprobe), dtype=torch.int32, device=queries.device)
+        pd = torch.empty((nq, nprobe), dtype=torch.float32, device=queries.device)
+    else:
+        pid, pd = out
+    _check(load_library().ivfpq_probe_static(ix.handle, queries.data_ptr(), nq, nprobe, pid.data_ptr(),
+                                             pd.data_ptr(), _stream()), "ivfpq_probe_static")
+    return pid, pd

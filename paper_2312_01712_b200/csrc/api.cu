@@ -380,6 +380,7 @@ const char* ivfpq_error_string(int code) {
         case IVFPQ_ERR_WORKSPACE: return "workspace or derived buffer too small or misaligned";
         case IVFPQ_ERR_CUDA: return "CUDA runtime error";
         case IVFPQ_ERR_DEVICE_FLAG: return "device-side status flag raised";
+        case IVFPQ_ERR_STATIC_LIMIT: return "index too large for the scratch array built into the library";
         default: return "unknown error code";
     }
 }

@@ -5,6 +5,8 @@
 // per dimension, j ascending, fp32: the selection must reproduce the defining arithmetic bit for
 // bit, and the GEMM form |c|^2 - 2 q.c + |q|^2 that the paper uses on tensor cores (Sec. 4.3,
 // last paragraph) rounds differently near the nprobe-th distance.
+#include <mutex>
+
 #include "common.cuh"
 #include "topk.cuh"
 
@@ -120,4 +122,60 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------------------------
+// Filtering stage without any caller-provided or allocated scratch (ivfpq_probe_static).
+//
+// The [queries][nlist] distance tile that coarse_dist_kernel writes and select_probes_kernel reads
+// lives in a fixed array inside the library image.  Every GPU that loads the library carries these
+// bytes until the process exits; all calls on a device share them.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// first 256 bytes: device status word (cleared by every call); the rest: the distance tile
+static __device__ __align__(256) unsigned char g_static_scratch[IVFPQ_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};  // device address of g_static_scratch, per device ordinal
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can
+// use: the device address has to be asked for, once per device, with that device current.
+int static_scratch_address(int device, unsigned char** out) {
+    if (device < 0 || device >= kMaxDevices) return IVFPQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[device]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return IVFPQ_ERR_CUDA;
+        g_static_ptr[device] = p;
+    }
+    *out = static_cast<unsigned char*>(g_static_ptr[device]);
+    return IVFPQ_OK;
+}
+
+}  // namespace
+
 }  // namespace ivfpq
+
+extern "C" int ivfpq_probe_static(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
+                                  int32_t* probe_ids, float* probe_d, void* stream) {
+    if (!index || !queries || !probe_ids || !probe_d) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (nq <= 0 || nprobe <= 0) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (nprobe > index->nlist || nprobe > IVFPQ_MAX_NPROBE || nq > (int64_t)1 << 24) return IVFPQ_ERR_UNSUPPORTED;
+    if (index->nlist > IVFPQ_STATIC_MAX_NLIST) return IVFPQ_ERR_STATIC_LIMIT;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    if (dev != index->device) return IVFPQ_ERR_INVALID_ARGUMENT;  // the index lives on another GPU
+    unsigned char* scratch = nullptr;
+    const int rc = ivfpq::static_scratch_address(dev, &scratch);
+    if (rc != IVFPQ_OK) return rc;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // the status word must start at zero; the tile is fully rewritten before it is read
+    if (cudaMemsetAsync(scratch, 0, 256, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    int64_t qchunk = ((int64_t)IVFPQ_STATIC_SCRATCH_BYTES - 256) / ((int64_t)index->nlist * 4);
+    if (qchunk > nq) qchunk = nq;
+    int64_t launches = 0;
+    if (ivfpq::launch_coarse(index, queries, nq, nprobe, reinterpret_cast<float*>(scratch + 256), qchunk,
+                             probe_ids, probe_d, reinterpret_cast<int*>(scratch), st, &launches) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    return IVFPQ_OK;
+}
