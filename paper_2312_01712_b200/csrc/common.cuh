@@ -53,6 +53,9 @@ struct ivfpq_index {
 
 namespace ivfpq {
 
+// Shape served by the persistent kernel (scan_pers.cu); its code layout is the additive rotation.
+inline bool pers_shape(const ivfpq_index* ix) { return ix->rot && ix->nsub == 16 && ix->dsub == 8; }
+
 struct SearchArgs {
     const ivfpq_index* ix;
     const float* queries;     // dev [nq][d]

@@ -336,7 +336,7 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     const size_t smem = scan_smem_bytes(ix->nw, ix->d, a.nprobe, a.debug);
     const int64_t grid = a.nq * sp.nsplit;
     cudaError_t e;
-    if (ix->rot && ix->nsub == 16 && ix->dsub == 8)
+    if (pers_shape(ix))
         e = launch_scan_pers(ix, sp, grid, a.debug, a.nprobe, st);
     else if (ix->rot)
         e = launch_scan_rot(ix, sp, grid, a.debug, a.nprobe, st);

@@ -340,7 +340,6 @@ bool rot_supported(int nsub, int dsub) {
 
 cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, bool debug, int nprobe,
                             cudaStream_t st) {
-    if (ix->nsub == 16 && ix->dsub == 8) return launch_rot<16, 0, 0, 8, 256>(sp, grid, debug, nprobe, st);
     if (ix->nsub == 48 && ix->dsub == 2) return launch_rot<32, 16, 0, 2, 256>(sp, grid, debug, nprobe, st);
     if (ix->nsub == 50 && ix->dsub == 4) return launch_rot<32, 16, 2, 4, 256>(sp, grid, debug, nprobe, st);
     if (ix->nsub == 8 && ix->dsub == 4) return launch_rot<8, 0, 0, 4, 256>(sp, grid, debug, nprobe, st);
