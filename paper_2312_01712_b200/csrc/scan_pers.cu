@@ -21,8 +21,11 @@
 //     different warps overlap on the SM;
 //   * list metadata of the item's clusters is staged in shared memory once per item; the first
 //     code blocks of a list are requested before the table build and arrive during it;
-//   * candidates go to the CTA's streaming top-k; a warp checks a soft fill limit before every
-//     block and the CTA compacts only when that limit was hit.
+//   * candidates go to the CTA's candidate buffer as (distance, position in the id array): the
+//     id itself is read only when the buffer is compacted, for all new candidates at once, so
+//     the scan loop never waits for that load.  A warp checks a soft fill limit before every block
+//     and the CTA compacts only when that limit was hit, with one histogram pass over the
+//     distances (topk.cuh); the final k are ranked by counting and written straight to the output.
 #include "common.cuh"
 #include "scan_common.cuh"
 #include "topk.cuh"
@@ -56,7 +59,7 @@ __host__ __device__ inline int pers_aux_bytes(int nprobe, bool dbg) {
     b += kMetaCap * (int)sizeof(ProbeMeta);
     b += kW * kDsub * 4;                  // query
     b += 64 * 4;                          // squared thresholds (padded)
-    b += 32 + kTopkHistInts * 4;          // threshold, counters, selection histogram
+    b += 32 + (kNT + kQuickExtra) * 4;    // threshold, counters, compaction histogram
     if (dbg) b += 2 * kW * 8 * 4 + (nprobe + 1) * 8;
     return (b + 255) & ~255;
 }
@@ -103,6 +106,20 @@ __device__ __forceinline__ float gather16(const uint4 cur, uint32_t bsel) {
     return a0 + a1;
 }
 
+// The keys pushed since the last compaction carry the position of the point in the id array;
+// replace it by the id (equal distances are ordered by id).  Called by all threads after a
+// barrier that follows the last push; the first *ntrans keys already hold ids.
+__device__ __forceinline__ void translate_new_keys(const TopkState& t, const int* ntrans,
+                                                   const int32_t* __restrict__ ids) {
+    const int n = min(*t.cnt, kTopkCap);
+    for (int i = *ntrans + threadIdx.x; i < n; i += kNT) {
+        const unsigned long long key = t.buf[i];
+        const uint32_t id = (uint32_t)__ldg(ids + (uint32_t)(key & 0xFFFFFFFFull));
+        t.buf[i] = (key & 0xFFFFFFFF00000000ull) | id;
+    }
+    // the compaction that follows starts with a barrier
+}
+
 template <bool DBG>
 __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams p, const int64_t nitems) {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -128,8 +145,9 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
     float* r2 = qs + d;
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + 64);
     int* cnt_p = reinterpret_cast<int*>(tau_p + 1);
-    int* hist_p = reinterpret_cast<int*>(tau_p + 4);
-    uint32_t* hitmask = reinterpret_cast<uint32_t*>(hist_p + kTopkHistInts);     // DBG only: [2][16][8]
+    int* ntrans_p = cnt_p + 1;                                                   // keys that already hold ids
+    int* hist_p = reinterpret_cast<int*>(tau_p + 4);                             // [kNT + kQuickExtra]
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(hist_p + kNT + kQuickExtra);     // DBG only: [2][16][8]
     long long* vprefix = reinterpret_cast<long long*>(hitmask + 2 * kW * 8);     // DBG only
     TopkState t{kbuf, cnt_p, tau_p, hist_p};
 
@@ -184,6 +202,8 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
         r[6] = __fsub_rn(b.z, cv[6]); r[7] = __fsub_rn(b.w, cv[7]);
     };
 
+    topk_quick_init<kNT>(hist_p);
+
     for (int64_t item = blockIdx.x; item < nitems; item += gridDim.x) {
         const int64_t q = item / p.nsplit;
         const int split = (int)(item % p.nsplit);
@@ -210,6 +230,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
             vprefix[p.nprobe] = run;
             if (p.visit_count) p.visit_count[q] = run;
         }
+        if (tid == 0) *ntrans_p = 0;
         topk_init(t);  // contains a barrier
         float P = 0.0f;
         if (!p.dense) {
@@ -296,8 +317,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
                 const uint32_t bsel = (lut_win + (uint32_t)(j & 1) * kLutBytes) | (uint32_t)(lane * 4);
                 const uint32_t* hm = hitmask + (j & 1) * kW * 8;
                 while (true) {
-                    const unsigned long long tau = *tau_p;
-                    const uint32_t tau_hi = (uint32_t)(tau >> 32);
+                    const uint32_t tau_hi = (uint32_t)(*tau_p >> 32);
                     while (blk < nblk) {
                         if (*reinterpret_cast<volatile int*>(cnt_p) >= kSoftLimit) break;
                         const uint4 cur = n0;
@@ -322,11 +342,11 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
                                     if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[m.p0 + pos];
                                 }
                             }
+                            // distance-only test: a tie with the threshold distance is sorted out
+                            // at the next compaction, once the id is known
                             if (__float_as_uint(acc) <= tau_hi) {
-                                const unsigned long long key = make_key(acc, (uint32_t)p.ids[m.p0 + pos]);
-                                if (key < tau) {
-                                    if (!topk_push(t, key)) atomicOr(p.status, kFlagOverflow);
-                                }
+                                if (!topk_push(t, make_key(acc, (uint32_t)(m.p0 + pos))))
+                                    atomicOr(p.status, kFlagOverflow);
                             }
                         }
                         blk += kWarps;
@@ -334,22 +354,33 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
                     // the barrier that separates cluster j from cluster j + 1 (table j + 1 complete,
                     // table j free); a set flag means some warp stopped at the soft limit
                     if (!__syncthreads_or(blk < nblk)) break;
-                    topk_select<kNT>(t, p.k);
+                    translate_new_keys(t, ntrans_p, p.ids);
+                    topk_quick_compact<kNT>(t, p.k, hist_p);
+                    if (tid == 0) *ntrans_p = *cnt_p;  // read again only after later barriers
                 }
             }
         }
 
-        topk_finalize<kNT>(t, p.k);
-        const int n = *cnt_p;
+        // ---- the exact k smallest (distance, id), ascending (paper Sec. 2.1, last paragraph) ----
+        translate_new_keys(t, ntrans_p, p.ids);
+        topk_quick_compact<kNT>(t, p.k, hist_p);   // leaves k or a few more keys; starts with a barrier
+        __syncthreads();
+        const int n = min(*cnt_p, kTopkCap);
         if (p.nsplit == 1) {
-            for (int i = tid; i < p.k; i += kNT) {
-                const unsigned long long key = i < n ? kbuf[i] : kKeyPad;
-                p.out_dist[q * p.k + i] = __uint_as_float((uint32_t)(key >> 32));
-                p.out_ids[q * p.k + i] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
+            float* od = p.out_dist + q * p.k;
+            int32_t* oi = p.out_ids + q * p.k;
+            topk_emit_ranked<kNT>(t, n, p.k, [&](int rank, unsigned long long key) {
+                od[rank] = __uint_as_float((uint32_t)(key >> 32));
+                oi[rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
+            });
+            for (int i = n + tid; i < p.k; i += kNT) {
+                od[i] = __uint_as_float((uint32_t)(kKeyPad >> 32));
+                oi[i] = -1;
             }
         } else {
             unsigned long long* dst = p.partial + (q * p.nsplit + split) * p.k;
-            for (int i = tid; i < p.k; i += kNT) dst[i] = i < n ? kbuf[i] : kKeyPad;
+            topk_emit_ranked<kNT>(t, n, p.k, [&](int rank, unsigned long long key) { dst[rank] = key; });
+            for (int i = n + tid; i < p.k; i += kNT) dst[i] = kKeyPad;
         }
     }
 }

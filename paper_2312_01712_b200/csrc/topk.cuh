@@ -174,4 +174,151 @@ __device__ __forceinline__ void topk_round_end(const TopkState& t, int k, int ne
     if (c + next_items > kTopkCap) topk_select<NT>(t, k);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Quick compaction and ranked output (used by the persistent scan kernel).
+//
+// Between two compactions any valid threshold will do, so the buffer is not reduced to exactly
+// k keys: one histogram pass over the distance bits (NT bins spread evenly between the smallest
+// and the largest buffered distance) finds the first bin boundary below which at least k keys
+// lie; those keys are kept and the boundary becomes the threshold.  Only the final answer is
+// exact: the few survivors are ranked by counting, for each key, the keys below it, and written
+// straight to their output slots.
+//
+// `qs` is an int array of NT + kQuickExtra words of shared memory that is all zero between calls
+// except qs[NT] (running minimum, kept at 0xFFFFFFFF): topk_quick_init sets this up once.
+// ---------------------------------------------------------------------------------------------
+constexpr int kQuickExtra = 40;  // words behind the NT bins: min, max, result (2), warp sums (32)
+
+template <int NT>
+__device__ __forceinline__ void topk_quick_init(int* qs) {
+    for (int i = threadIdx.x; i < NT + kQuickExtra; i += NT) qs[i] = (i == NT) ? -1 : 0;
+    __syncthreads();
+}
+
+// Keeps the keys below a bin boundary chosen so that at least k survive; sets the threshold to
+// that boundary.  No-op when at most k keys are buffered.  Falls back to the exact selection when
+// the histogram cannot separate the distances (e.g. all equal).  Must be called by all threads;
+// contains barriers.
+template <int NT>
+__device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
+    constexpr int kPerThread = (kTopkCap + NT - 1) / NT;
+    static_assert(NT >= 64 && NT <= 1024 && (NT & (NT - 1)) == 0, "one bin per thread, power of two");
+    __syncthreads();
+    const int n = min(*t.cnt, kTopkCap);
+    if (n <= k) return;  // uniform over the CTA
+    const int tid = threadIdx.x;
+    unsigned* uq = reinterpret_cast<unsigned*>(qs);
+    unsigned long long mine[kPerThread];
+    unsigned lo = 0xFFFFFFFFu, hi = 0u;
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+        const int i = tid + j * NT;
+        mine[j] = i < n ? t.buf[i] : ~0ull;
+        if (i < n) {
+            const unsigned h = (unsigned)(mine[j] >> 32);
+            lo = min(lo, h);
+            hi = max(hi, h);
+        }
+    }
+    lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+    if ((tid & 31) == 0) {
+        atomicMin(&uq[NT], lo);
+        atomicMax(&uq[NT + 1], hi);
+    }
+    __syncthreads();
+    lo = uq[NT];
+    hi = uq[NT + 1];
+    const unsigned range = hi - lo;
+    int shift = 0;  // smallest shift with (range >> shift) < NT
+    if (range >= (unsigned)NT) shift = (32 - __clz(range)) - (31 - __clz(NT));
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+        const int i = tid + j * NT;
+        if (i < n) atomicAdd(&qs[((unsigned)(mine[j] >> 32) - lo) >> shift], 1);
+    }
+    __syncthreads();
+    // inclusive prefix sum over the NT bins, one bin per thread
+    const int v = qs[tid];
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if ((tid & 31) >= o) incl += x;
+    }
+    if ((tid & 31) == 31) qs[NT + 4 + (tid >> 5)] = incl;
+    __syncthreads();
+    int before = 0;
+    for (int w = 0; w < (tid >> 5); ++w) before += qs[NT + 4 + w];
+    incl += before;
+    if (incl - v < k && k <= incl) {  // exactly one thread: its bin holds the k-th smallest distance
+        qs[NT + 2] = tid;
+        qs[NT + 3] = incl;
+    }
+    __syncthreads();
+    const int bstar = qs[NT + 2];
+    const int kept = qs[NT + 3];
+    __syncthreads();  // everybody has read the result and the warp sums
+    qs[tid] = 0;      // back to the all-zero state for the next call
+    if (tid < kQuickExtra) qs[NT + tid] = (tid == 0) ? -1 : 0;
+    if (kept >= n) {  // uniform: nothing would be dropped
+        __syncthreads();
+        topk_select<NT>(t, k);  // uses the same shared words as its histogram
+        topk_quick_init<NT>(qs);
+        return;
+    }
+    // exclusive bound on the keys that stay
+    const unsigned long long bound = ((unsigned long long)lo + ((unsigned long long)(bstar + 1) << shift)) << 32;
+    if (tid == 0) {
+        *t.cnt = 0;
+        *t.tau = bound < kKeyPad ? bound : kKeyPad;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+        const bool keep = mine[j] < bound;  // the filler ~0 never passes
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, keep);
+        if (bal != 0) {
+            int base = 0;
+            if ((tid & 31) == 0) base = atomicAdd(t.cnt, __popc(bal));
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            if (keep) t.buf[base + __popc(bal & ((1u << (tid & 31)) - 1u))] = mine[j];
+        }
+    }
+    __syncthreads();
+}
+
+// Rank of every buffered key among the n buffered keys (n <= kTopkCap), by counting; calls
+// emit(rank, key) for the keys of rank < k.  Equal keys are ordered by buffer position, so ranks
+// are distinct.  All threads must call it; the buffer must be complete (barrier before).
+template <int NT, class Emit>
+__device__ __forceinline__ void topk_emit_ranked(const TopkState& t, int n, int k, Emit emit) {
+    const int tid = threadIdx.x;
+    if (n * 2 <= NT) {
+        // G consecutive lanes share a key and split the comparisons
+        int G = 2;
+        while (G < 32 && n * (G * 2) <= NT) G *= 2;
+        const int i = tid / G, part = tid & (G - 1);
+        int rank = 0;
+        const unsigned long long me = i < n ? t.buf[i] : 0ull;
+        if (i < n)
+            for (int j = part; j < n; j += G) {
+                const unsigned long long o = t.buf[j];
+                rank += (o < me || (o == me && j < i)) ? 1 : 0;
+            }
+        for (int o = 1; o < G; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+        if (i < n && part == 0 && rank < k) emit(rank, me);
+    } else {
+        for (int i = tid; i < n; i += NT) {
+            const unsigned long long me = t.buf[i];
+            int rank = 0;
+            for (int j = 0; j < n; ++j) {
+                const unsigned long long o = t.buf[j];
+                rank += (o < me || (o == me && j < i)) ? 1 : 0;
+            }
+            if (rank < k) emit(rank, me);
+        }
+    }
+}
+
 }  // namespace ivfpq
