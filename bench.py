@@ -40,6 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one scan-kernel launch, from the ncu captures
 # summarised under profiles/ (bytes per launch of the benchmark's workload; None = not captured).
 SCAN_DRAM_TRAFFIC_BYTES = {}
+SCAN_KERNEL = {1608: "scan_ws16x8_kernel"}
 
 
 def log(*a):
@@ -272,6 +273,11 @@ def run_cuda(args):
     scan_ms = float(np.mean([s[1] for s in stages]))
     coarse_ms = float(np.mean([s[0] for s in stages]))
     achieved = scan_bytes / (scan_ms * 1e-3) / 1e9
+    # shared-memory ceiling of the scan: one conflict-free 32-lane table gather per SM per clock
+    props = torch.cuda.get_device_properties(local_rank)
+    clk = sampler.summary()["sm_mhz"] or sampler.summary()["sm_max_mhz"] or 1965.0
+    gather_peak = props.multi_processor_count * 32 * clk * 1e6 / 1e9            # G gathers/s
+    gather_rate = scan_bytes / (scan_ms * 1e-3) / 1e9                            # one gather per code byte
 
     cpu = cpu_baseline(index, q_np, nprobe, k, radius, scale, args.cpu_sample)
 
@@ -294,10 +300,14 @@ def run_cuda(args):
                 "h2d_bytes_per_step": int(qh.numel() * 4), "d2h_bytes_per_step": int(odh.numel() * 4 + oih.numel() * 4)},
         "gpu_launches": int(launches),
         "clocks": sampler.summary(),
-        "roofline": {"bound": "hbm", "kernel": "scan_kernel (selective LUT + list scan + top-k)",
+        "roofline": {"bound": "hbm", "kernel": SCAN_KERNEL.get(index.nsub * 100 + index.dsub, "scan_rot_kernel") +
+                     " (selective LUT + list scan + top-k)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": f"of {peak_src}", "algorithmic_bytes_per_launch": int(scan_bytes),
                      "visits_per_launch": int(visits), "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload)},
+        "gather_roofline": {"bound": "shared-memory gathers", "achieved": gather_rate, "peak": gather_peak,
+                            "unit": "Ggather/s", "frac": gather_rate / gather_peak,
+                            "peak_source": f"{props.multi_processor_count} SMs x 32 lanes x {clk:.0f} MHz"},
         "cpu_baseline": cpu,
     }
     print(json.dumps(line), flush=True)

@@ -2,6 +2,7 @@
 // See include/ivfpq.h for the contract of every entry point.
 #include <math.h>
 #include <new>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -197,6 +198,10 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->vec16 = dl.vec16;
     ix->nblocks = dl.nblocks;
     ix->rot = dl.rot;
+    {
+        const char* kind = getenv("IVFPQ_PERS_KIND");
+        ix->pers_kind = (kind && kind[0] == '2') ? 2 : 1;
+    }
     for (int i = 0; i < 3; ++i) ix->gw[i] = dl.rot ? dl.gw[i] : 0;
     ix->block_bytes = dl.block_bytes;
     ix->cbt = reinterpret_cast<const float*>(base + dl.cbt_off);

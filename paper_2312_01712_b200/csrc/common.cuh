@@ -15,6 +15,8 @@ constexpr int kTopkCap = 2048;       // candidate buffer slots per CTA (>= IVFPQ
 // Device status bits (workspace status word).
 constexpr int kFlagBadList = 1;   // a probed cluster id or code block was out of range and was skipped
 constexpr int kFlagOverflow = 2;  // the candidate buffer would have overflowed; the candidate was dropped
+constexpr int kFlagTimeout = 4;   // a bounded wait between cooperating warps ran out
+constexpr int kFlagLayout = 8;    // the kernel's shared-memory layout does not fit the window offset it was given
 
 inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -36,6 +38,7 @@ struct ivfpq_index {
     int64_t nblocks;          // total 32-point blocks
     // rotated layout (scan_rot.cu): subspace groups of power-of-two width, codes stored per lane in
     // the lane's own visiting order, codebook copied entry-major per group
+    int32_t pers_kind;        // 16 x 8 shape: 1 = scan_pers.cu (additive rotation), 2 = scan_ws.cu (xor rotation)
     int32_t rot;              // 1: rotated layout in use
     int32_t gw[3];            // group widths, largest first, 0 = unused
     int32_t block_bytes;      // bytes of one 32-point code block in the rotated layout

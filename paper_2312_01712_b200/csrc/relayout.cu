@@ -122,7 +122,7 @@ cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_
         if (ix->nblocks > 0)
             relayout_rot_kernel<<<ix->nlist, 256, 0, st>>>(codes, ix->list_off, ix->list_blk, ix->nsub, ix->gw[0],
                                                            ix->gw[1], ix->gw[2], ix->block_bytes,
-                                                           pers_shape(ix) ? 1 : 0,
+                                                           (pers_shape(ix) && ix->pers_kind == 1) ? 1 : 0,
                                                            reinterpret_cast<unsigned char*>(codes_il));
         relayout_cbt_kernel<<<64, 256, 0, st>>>(ix->cb, ix->nsub, ix->dsub, ix->ksub, ix->gw[0], ix->gw[1],
                                                 ix->gw[2], cbt);

@@ -59,7 +59,7 @@ __host__ __device__ inline int pers_aux_bytes(int nprobe, bool dbg) {
     b += kMetaCap * (int)sizeof(ProbeMeta);
     b += kW * kDsub * 4;                  // query
     b += 64 * 4;                          // squared thresholds (padded)
-    b += 32 + (kNT + kQuickExtra) * 4;    // threshold, counters, compaction histogram
+    b += 32 + kQuickWords * 4;    // threshold, counters, compaction histogram
     if (dbg) b += 2 * kW * 8 * 4 + (nprobe + 1) * 8;
     return (b + 255) & ~255;
 }
@@ -146,8 +146,8 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + 64);
     int* cnt_p = reinterpret_cast<int*>(tau_p + 1);
     int* ntrans_p = cnt_p + 1;                                                   // keys that already hold ids
-    int* hist_p = reinterpret_cast<int*>(tau_p + 4);                             // [kNT + kQuickExtra]
-    uint32_t* hitmask = reinterpret_cast<uint32_t*>(hist_p + kNT + kQuickExtra);     // DBG only: [2][16][8]
+    int* hist_p = reinterpret_cast<int*>(tau_p + 4);                             // [kQuickWords]
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(hist_p + kQuickWords);     // DBG only: [2][16][8]
     long long* vprefix = reinterpret_cast<long long*>(hitmask + 2 * kW * 8);     // DBG only
     TopkState t{kbuf, cnt_p, tau_p, hist_p};
 
@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
         if (p.nsplit == 1) {
             float* od = p.out_dist + q * p.k;
             int32_t* oi = p.out_ids + q * p.k;
-            topk_emit_ranked<kNT>(t, n, p.k, [&](int rank, unsigned long long key) {
+            topk_emit_ranked<kNT, CtaGroup>(t, n, p.k, [&](int rank, unsigned long long key) {
                 od[rank] = __uint_as_float((uint32_t)(key >> 32));
                 oi[rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
             });
@@ -379,7 +379,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
             }
         } else {
             unsigned long long* dst = p.partial + (q * p.nsplit + split) * p.k;
-            topk_emit_ranked<kNT>(t, n, p.k, [&](int rank, unsigned long long key) { dst[rank] = key; });
+            topk_emit_ranked<kNT, CtaGroup>(t, n, p.k, [&](int rank, unsigned long long key) { dst[rank] = key; });
             for (int i = n + tid; i < p.k; i += kNT) dst[i] = kKeyPad;
         }
     }

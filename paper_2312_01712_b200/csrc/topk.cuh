@@ -18,6 +18,13 @@ namespace ivfpq {
 constexpr unsigned long long kKeyPad = 0x7F800000FFFFFFFFull;  // (+inf, id -1): sorts after every real key
 constexpr int kTopkHistInts = 264;                             // 256 bins + 3 result words, padded
 
+// Which threads cooperate in a selection: the whole CTA by default; a kernel whose warps have
+// different roles passes a policy with its own thread numbering and named barrier.
+struct CtaGroup {
+    __device__ __forceinline__ static int tid() { return threadIdx.x; }
+    __device__ __forceinline__ static void sync() { __syncthreads(); }
+};
+
 struct TopkState {
     unsigned long long* buf;  // [kTopkCap] shared memory
     int* cnt;                 // shared
@@ -70,19 +77,19 @@ __device__ inline void bitonic_sort(unsigned long long* buf, int n2) {
 
 // Keeps the k smallest keys of the buffer (unordered) and sets the threshold to an exclusive
 // upper bound of the kept keys.  No-op when at most k keys are buffered.  NT = threads per CTA.
-template <int NT>
+template <int NT, class G = CtaGroup>
 __device__ inline void topk_select(const TopkState& t, int k) {
     constexpr int kPerThread = (kTopkCap + NT - 1) / NT;
-    __syncthreads();
+    G::sync();
     const int n = min(*t.cnt, kTopkCap);
     if (n <= k) return;  // uniform over the CTA
-    const int tid = threadIdx.x;
+    const int tid = G::tid();
     unsigned long long prefix = 0;  // high digits of the k-th smallest key found so far
     int need = k;                   // rank of the wanted key among the keys that share the prefix
     int shift = 56;
     for (;; shift -= 8) {
         for (int i = tid; i < 256; i += NT) t.hist[i] = 0;
-        __syncthreads();
+        G::sync();
         for (int i0 = 0; i0 < n; i0 += NT) {  // whole warps iterate together (warp-aggregated counting)
             const int i = i0 + tid;
             int digit = -1;
@@ -94,7 +101,7 @@ __device__ inline void topk_select(const TopkState& t, int k) {
             const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
             if (digit >= 0 && (tid & 31) == __ffs(peers) - 1) atomicAdd(&t.hist[digit], __popc(peers));
         }
-        __syncthreads();
+        G::sync();
         if (tid < 32) {  // first warp: locate the bin that holds rank `need`
             int local[8], sum = 0;
 #pragma unroll
@@ -122,7 +129,7 @@ __device__ inline void topk_select(const TopkState& t, int k) {
                 }
             }
         }
-        __syncthreads();
+        G::sync();
         const int digit = t.hist[256], below = t.hist[257], inbin = t.hist[258];
         prefix |= (unsigned long long)digit << shift;
         need -= below;
@@ -138,16 +145,16 @@ __device__ inline void topk_select(const TopkState& t, int k) {
         mine[j] = i < n ? t.buf[i] : ~0ull;
         keep[j] = mine[j] < bound;
     }
-    __syncthreads();
+    G::sync();
     if (tid == 0) {
         *t.cnt = 0;
         *t.tau = bound;
     }
-    __syncthreads();
+    G::sync();
 #pragma unroll
     for (int j = 0; j < kPerThread; ++j)
         if (keep[j]) t.buf[atomicAdd(t.cnt, 1)] = mine[j];
-    __syncthreads();
+    G::sync();
 }
 
 // Final ordering: the k smallest keys, ascending, in buf[0..min(cnt, k)).
@@ -175,38 +182,41 @@ __device__ __forceinline__ void topk_round_end(const TopkState& t, int k, int ne
 }
 
 // ---------------------------------------------------------------------------------------------
-// Quick compaction and ranked output (used by the persistent scan kernel).
+// Quick compaction and ranked output (used by the persistent scan kernels).
 //
 // Between two compactions any valid threshold will do, so the buffer is not reduced to exactly
-// k keys: one histogram pass over the distance bits (NT bins spread evenly between the smallest
-// and the largest buffered distance) finds the first bin boundary below which at least k keys
-// lie; those keys are kept and the boundary becomes the threshold.  Only the final answer is
-// exact: the few survivors are ranked by counting, for each key, the keys below it, and written
-// straight to their output slots.
+// k keys: one histogram pass over the distance bits (kQuickBins bins spread evenly between the
+// smallest and the largest buffered distance) finds the first bin boundary below which at least
+// k keys lie; those keys are kept and the boundary becomes the threshold.  Only the final answer
+// is exact: the few survivors are ranked by counting, for each key, the keys below it, and
+// written straight to their output slots.
 //
-// `qs` is an int array of NT + kQuickExtra words of shared memory that is all zero between calls
-// except qs[NT] (running minimum, kept at 0xFFFFFFFF): topk_quick_init sets this up once.
+// `qs` is an int array of kQuickWords words of shared memory that is all zero between calls
+// except qs[kQuickBins] (running minimum, kept at 0xFFFFFFFF): topk_quick_init sets this up.
+// NT = threads of the group G (at least kQuickBins, whole warps).
 // ---------------------------------------------------------------------------------------------
-constexpr int kQuickExtra = 40;  // words behind the NT bins: min, max, result (2), warp sums (32)
+constexpr int kQuickBins = 256;
+constexpr int kQuickWords = kQuickBins + 40;  // + min, max, result (2), warp sums (up to 32)
 
-template <int NT>
+template <int NT, class G = CtaGroup>
 __device__ __forceinline__ void topk_quick_init(int* qs) {
-    for (int i = threadIdx.x; i < NT + kQuickExtra; i += NT) qs[i] = (i == NT) ? -1 : 0;
-    __syncthreads();
+    for (int i = G::tid(); i < kQuickWords; i += NT) qs[i] = (i == kQuickBins) ? -1 : 0;
+    G::sync();
 }
 
 // Keeps the keys below a bin boundary chosen so that at least k survive; sets the threshold to
 // that boundary.  No-op when at most k keys are buffered.  Falls back to the exact selection when
-// the histogram cannot separate the distances (e.g. all equal).  Must be called by all threads;
-// contains barriers.
-template <int NT>
+// the histogram cannot separate the distances (e.g. all equal).  Must be called by all threads of
+// the group; contains barriers.
+template <int NT, class G = CtaGroup>
 __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
     constexpr int kPerThread = (kTopkCap + NT - 1) / NT;
-    static_assert(NT >= 64 && NT <= 1024 && (NT & (NT - 1)) == 0, "one bin per thread, power of two");
-    __syncthreads();
+    constexpr int B = kQuickBins;
+    static_assert(NT >= B && NT % 32 == 0, "one bin per thread of the first B threads");
+    G::sync();
     const int n = min(*t.cnt, kTopkCap);
-    if (n <= k) return;  // uniform over the CTA
-    const int tid = threadIdx.x;
+    if (n <= k) return;  // uniform over the group
+    const int tid = G::tid();
     unsigned* uq = reinterpret_cast<unsigned*>(qs);
     unsigned long long mine[kPerThread];
     unsigned lo = 0xFFFFFFFFu, hi = 0u;
@@ -223,48 +233,50 @@ __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
     lo = __reduce_min_sync(0xFFFFFFFFu, lo);
     hi = __reduce_max_sync(0xFFFFFFFFu, hi);
     if ((tid & 31) == 0) {
-        atomicMin(&uq[NT], lo);
-        atomicMax(&uq[NT + 1], hi);
+        atomicMin(&uq[B], lo);
+        atomicMax(&uq[B + 1], hi);
     }
-    __syncthreads();
-    lo = uq[NT];
-    hi = uq[NT + 1];
+    G::sync();
+    lo = uq[B];
+    hi = uq[B + 1];
     const unsigned range = hi - lo;
-    int shift = 0;  // smallest shift with (range >> shift) < NT
-    if (range >= (unsigned)NT) shift = (32 - __clz(range)) - (31 - __clz(NT));
+    int shift = 0;  // smallest shift with (range >> shift) < B
+    if (range >= (unsigned)B) shift = (32 - __clz(range)) - (31 - __clz(B));
 #pragma unroll
     for (int j = 0; j < kPerThread; ++j) {
         const int i = tid + j * NT;
         if (i < n) atomicAdd(&qs[((unsigned)(mine[j] >> 32) - lo) >> shift], 1);
     }
-    __syncthreads();
-    // inclusive prefix sum over the NT bins, one bin per thread
-    const int v = qs[tid];
+    G::sync();
+    // inclusive prefix sum over the bins, one bin per thread of the first B threads
+    const int v = tid < B ? qs[tid] : 0;
     int incl = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const int x = __shfl_up_sync(0xFFFFFFFFu, incl, o);
         if ((tid & 31) >= o) incl += x;
     }
-    if ((tid & 31) == 31) qs[NT + 4 + (tid >> 5)] = incl;
-    __syncthreads();
-    int before = 0;
-    for (int w = 0; w < (tid >> 5); ++w) before += qs[NT + 4 + w];
-    incl += before;
-    if (incl - v < k && k <= incl) {  // exactly one thread: its bin holds the k-th smallest distance
-        qs[NT + 2] = tid;
-        qs[NT + 3] = incl;
+    if (tid < B && (tid & 31) == 31) qs[B + 4 + (tid >> 5)] = incl;
+    G::sync();
+    if (tid < B) {
+        int before = 0;
+        for (int w = 0; w < (tid >> 5); ++w) before += qs[B + 4 + w];
+        incl += before;
+        if (incl - v < k && k <= incl) {  // exactly one thread: its bin holds the k-th smallest distance
+            qs[B + 2] = tid;
+            qs[B + 3] = incl;
+        }
     }
-    __syncthreads();
-    const int bstar = qs[NT + 2];
-    const int kept = qs[NT + 3];
-    __syncthreads();  // everybody has read the result and the warp sums
-    qs[tid] = 0;      // back to the all-zero state for the next call
-    if (tid < kQuickExtra) qs[NT + tid] = (tid == 0) ? -1 : 0;
+    G::sync();
+    const int bstar = qs[B + 2];
+    const int kept = qs[B + 3];
+    G::sync();  // everybody has read the result and the warp sums
+    if (tid < B) qs[tid] = 0;  // back to the all-zero state for the next call
+    if (tid < kQuickWords - B) qs[B + tid] = (tid == 0) ? -1 : 0;
     if (kept >= n) {  // uniform: nothing would be dropped
-        __syncthreads();
-        topk_select<NT>(t, k);  // uses the same shared words as its histogram
-        topk_quick_init<NT>(qs);
+        G::sync();
+        topk_select<NT, G>(t, k);  // uses the same shared words as its histogram
+        topk_quick_init<NT, G>(qs);
         return;
     }
     // exclusive bound on the keys that stay
@@ -273,7 +285,7 @@ __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
         *t.cnt = 0;
         *t.tau = bound < kKeyPad ? bound : kKeyPad;
     }
-    __syncthreads();
+    G::sync();
 #pragma unroll
     for (int j = 0; j < kPerThread; ++j) {
         const bool keep = mine[j] < bound;  // the filler ~0 never passes
@@ -285,28 +297,29 @@ __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
             if (keep) t.buf[base + __popc(bal & ((1u << (tid & 31)) - 1u))] = mine[j];
         }
     }
-    __syncthreads();
+    G::sync();
 }
 
 // Rank of every buffered key among the n buffered keys (n <= kTopkCap), by counting; calls
 // emit(rank, key) for the keys of rank < k.  Equal keys are ordered by buffer position, so ranks
-// are distinct.  All threads must call it; the buffer must be complete (barrier before).
-template <int NT, class Emit>
+// are distinct.  All threads of the group must call it; the buffer must be complete (barrier
+// before).
+template <int NT, class G = CtaGroup, class Emit>
 __device__ __forceinline__ void topk_emit_ranked(const TopkState& t, int n, int k, Emit emit) {
-    const int tid = threadIdx.x;
+    const int tid = G::tid();
     if (n * 2 <= NT) {
-        // G consecutive lanes share a key and split the comparisons
-        int G = 2;
-        while (G < 32 && n * (G * 2) <= NT) G *= 2;
-        const int i = tid / G, part = tid & (G - 1);
+        // S consecutive lanes share a key and split the comparisons
+        int S = 2;
+        while (S < 32 && n * (S * 2) <= NT) S *= 2;
+        const int i = tid / S, part = tid & (S - 1);
         int rank = 0;
         const unsigned long long me = i < n ? t.buf[i] : 0ull;
         if (i < n)
-            for (int j = part; j < n; j += G) {
+            for (int j = part; j < n; j += S) {
                 const unsigned long long o = t.buf[j];
                 rank += (o < me || (o == me && j < i)) ? 1 : 0;
             }
-        for (int o = 1; o < G; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+        for (int o = 1; o < S; o <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
         if (i < n && part == 0 && rank < k) emit(rank, me);
     } else {
         for (int i = tid; i < n; i += NT) {

@@ -281,5 +281,19 @@ def test_full_size_c1_all_queries():
     _full_size_parity("c1", 8, 1000, 1.0)
 
 
+def test_full_size_c3_sampled_queries():
+    _full_size_parity("c3", 16, 64, 1.0)
+
+
+def test_full_size_c4_sampled_queries():
+    _full_size_parity("c4", 32, 48, 1.0)
+
+
+def test_full_size_c5_sampled_queries():
+    """100 M points (1.6 GB of codes, built in streamed chunks on the GPU): the whole 10 k-query
+    batch in one call as the benchmark does, a sample of it checked against the oracle."""
+    _full_size_parity("c5", 32, 24, 1.0)
+
+
 def test_full_size_c2_sampled_queries():
     _full_size_parity("c2", 16, 128, 1.0)
