@@ -40,7 +40,6 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one scan-kernel launch, from the ncu captures
 # summarised under profiles/ (bytes per launch of the benchmark's workload; None = not captured).
 SCAN_DRAM_TRAFFIC_BYTES = {}
-SCAN_KERNEL = {1608: "scan_ws16x8_kernel"}
 
 
 def log(*a):
@@ -148,6 +147,15 @@ def pick_scale(search_sparse, search_dense, true_ids, scales=(0.5, 0.75, 1.0, 1.
         ids = search_sparse(float("inf"))
         chosen = (float("inf"), recall_at_k(ids, true_ids), recall_1_at_k(ids, true_ids))
     return r_dense, recall_1_at_k(dense_ids, true_ids), chosen, table
+
+
+def scan_kernel_name(index) -> str:
+    """Name of the kernel the library picks for this index (same rule as ivfpq_index_load)."""
+    if (index.nsub, index.dsub) == (16, 8):
+        forced = os.environ.get("IVFPQ_SCAN_KERNEL")
+        wide = forced == "wide" or (forced != "pers" and index.ntotal // index.nlist >= 2048)
+        return "scan_wide16x8_kernel" if wide else "scan_pers16x8_kernel"
+    return "scan_rot_kernel"
 
 
 def visits_per_batch(index, probe_ids: np.ndarray) -> int:
@@ -300,8 +308,7 @@ def run_cuda(args):
                 "h2d_bytes_per_step": int(qh.numel() * 4), "d2h_bytes_per_step": int(odh.numel() * 4 + oih.numel() * 4)},
         "gpu_launches": int(launches),
         "clocks": sampler.summary(),
-        "roofline": {"bound": "hbm", "kernel": SCAN_KERNEL.get(index.nsub * 100 + index.dsub, "scan_rot_kernel") +
-                     " (selective LUT + list scan + top-k)",
+        "roofline": {"bound": "hbm", "kernel": scan_kernel_name(index) + " (selective LUT + list scan + top-k)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": f"of {peak_src}", "algorithmic_bytes_per_launch": int(scan_bytes),
                      "visits_per_launch": int(visits), "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload)},

@@ -47,8 +47,8 @@ cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t
 cudaError_t launch_scan_pers(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
                              cudaStream_t st);
 
-// Warp-specialised persistent scan for the 16 x 8 quantizer (scan_ws.cu).
-cudaError_t launch_scan_ws(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
-                           cudaStream_t st);
+// 32-warp persistent scan for the 16 x 8 quantizer, codebook half in registers, half in shared memory (scan_wide.cu).
+cudaError_t launch_scan_wide(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
+                             cudaStream_t st);
 
 }  // namespace ivfpq

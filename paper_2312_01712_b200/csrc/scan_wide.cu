@@ -1,0 +1,466 @@
+// Persistent fused selective-LUT / list-scan / top-k kernel for the 16 x 8 product quantizer (16
+// subspaces of 8 dimensions, 256 entries), 32 warps per SM.  Same computation as scan.cu (paper
+// Sec. 2.1 steps B-D with the selection of Sec. 3.1 / Algorithm 2 and the miss constant of
+// Sec. 4.3).
+//
+//   * One CTA of 1024 threads per SM (64 registers per thread): eight warps per scheduler hide the
+//     latencies of the table gathers and of the code loads that four warps could not.
+//   * The 128 KB codebook stays on chip for the lifetime of the kernel, half in registers and half
+//     in shared memory: thread t owns subspace c = t & 15 and the entries u, u + 64, u + 128,
+//     u + 192 with u = t / 16; the first two live in its registers, the other two are read from
+//     shared memory (two 16-byte loads per entry, conflict-free).  Building a table reads nothing
+//     from global memory but the probed centroid (512 B, copied ahead with cp.async).
+//   * Table layout: 256 rows (entries) of 256 bytes; a row holds two tables side by side, 32
+//     columns each; column x holds the value of subspace x & 15 (two copies).  Lane l looks up, at
+//     step i, column l ^ i: the 32 lanes of a warp touch 32 different banks whatever the codes
+//     are.  The code bytes are stored in that visiting order when the index is loaded.  The table
+//     region sits at shared-window address 0x10000, so one byte-permute forms the address (byte 0:
+//     the lane's column offset for that step, byte 1: the code, bytes 2-3: zero) and the table base
+//     is the immediate of the load: three instructions per look-up.
+//   * Two tables: while the warps scan the list of cluster j they have already built their share of
+//     the table of cluster j + 1; one barrier per cluster separates the phases.
+//   * Code blocks: two per warp in registers, requested before the table build; further ahead the
+//     warp only asks for the lines to be brought into L2 (prefetch.global.L2, three blocks ahead
+//     and the first blocks of the next list), which keeps enough bytes in flight for lists that
+//     stream from HBM without spending registers.
+//   * Candidates go to the CTA's candidate buffer as (distance, position in the id array); ids are
+//     read when the buffer is compacted (one histogram pass, topk.cuh); the final k are ranked by
+//     counting and written straight to the output.
+#include <type_traits>
+
+#include "common.cuh"
+#include "scan_common.cuh"
+#include "topk.cuh"
+
+namespace ivfpq {
+
+namespace {
+
+constexpr int kW = 16;            // subspaces
+constexpr int kDsub = 8;
+constexpr int kD = kW * kDsub;
+constexpr int kNT = 1024;         // threads per CTA
+constexpr int kWarps = kNT / 32;
+constexpr int kEP = kNT / kW;     // entries per pass (64)
+constexpr int kNE = 256 / kEP;    // entries per thread (4): 0, 1 in registers, 2, 3 in shared memory
+constexpr int kRowBytes = 256;    // one table row (two tables side by side)
+constexpr uint32_t kLutWin = 0x10000;   // shared-window address of the table region (64 KB)
+constexpr uint32_t kCbWin = 0x20000;    // shared-window address of the shared half of the codebook (64 KB)
+constexpr int kCap = 4096;        // candidate buffer slots
+constexpr int kSoftLimit = 2048;  // compaction is requested once this many candidates are buffered
+constexpr int kMetaCap = 128;     // clusters whose metadata is staged at a time
+constexpr int kPfDist = 3;         // blocks (per warp) that the L2 prefetch runs ahead of the scan
+static_assert(kSoftLimit + kNT <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
+
+struct ProbeMeta {
+    long long b0;   // first 32-point code block of the list
+    int p0;         // first point of the list (index into ids; ntotal < 2^31)
+    int len;        // points in the list (0 when the cluster id or its tables were invalid)
+    int cl;         // cluster id, clamped into range
+    int pad;
+};
+
+// Auxiliary shared memory in front of the table region, in bytes.
+__host__ __device__ inline int wide_aux_bytes(int nprobe, bool dbg) {
+    int b = kCap * 8;                         // candidate keys
+    b += kMetaCap * (int)sizeof(ProbeMeta);
+    b += kD * 4 + 2 * kD * 4 + 64;            // query, two centroids, squared thresholds
+    b += 32 + kQuickWords * 4;                // threshold, counters, compaction histogram
+    if (dbg) b += 2 * kW * 8 * 4 + (nprobe + 1) * 8;
+    return (b + 255) & ~255;
+}
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(gsrc) : "memory");
+}
+// Asks for the 128-byte lines of the warp's addresses to be brought into L2 (no register, no wait).
+__device__ __forceinline__ void prefetch_l2(const void* gptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(gptr)); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// One table look-up.  `word` holds four code bytes, `pack` the lane's column offsets (lane ^ i) * 4
+// of the same four steps; T = byte of both that belongs to this step.  The permute builds
+// {0, 0, code, column offset} (the zero bytes are the replicated sign of the column offset, which is
+// below 128); the table base is the immediate.
+template <int T, int TABLE>
+__device__ __forceinline__ float lut_gather(uint32_t word, uint32_t pack) {
+    uint32_t addr;
+    float v;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(addr) : "r"(word), "r"(pack), "n"(((12 + T) << 12) | ((12 + T) << 8) | (T << 4) | (4 + T)));
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"((int)kLutWin + TABLE * 128) : "memory");
+    return v;
+}
+
+// Sum of the 16 table values of the lane's point.  Byte i of `cur` = code of subspace (lane ^ i) & 15.
+template <int TABLE>
+__device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[4]) {
+    float a0 = lut_gather<0, TABLE>(cur.x, pk[0]);
+    float a1 = lut_gather<1, TABLE>(cur.x, pk[0]);
+    a0 += lut_gather<2, TABLE>(cur.x, pk[0]);
+    a1 += lut_gather<3, TABLE>(cur.x, pk[0]);
+    a0 += lut_gather<0, TABLE>(cur.y, pk[1]);
+    a1 += lut_gather<1, TABLE>(cur.y, pk[1]);
+    a0 += lut_gather<2, TABLE>(cur.y, pk[1]);
+    a1 += lut_gather<3, TABLE>(cur.y, pk[1]);
+    a0 += lut_gather<0, TABLE>(cur.z, pk[2]);
+    a1 += lut_gather<1, TABLE>(cur.z, pk[2]);
+    a0 += lut_gather<2, TABLE>(cur.z, pk[2]);
+    a1 += lut_gather<3, TABLE>(cur.z, pk[2]);
+    a0 += lut_gather<0, TABLE>(cur.w, pk[3]);
+    a1 += lut_gather<1, TABLE>(cur.w, pk[3]);
+    a0 += lut_gather<2, TABLE>(cur.w, pk[3]);
+    a1 += lut_gather<3, TABLE>(cur.w, pk[3]);
+    return a0 + a1;
+}
+
+// The keys pushed since the last compaction carry the position of the point in the id array;
+// replace it by the id (equal distances are ordered by id).  Called by all threads after a
+// barrier that follows the last push; the first *ntrans keys already hold ids.
+__device__ __forceinline__ void translate_new_keys(const TopkState& t, const int* ntrans,
+                                                   const int32_t* __restrict__ ids) {
+    const int n = min(*t.cnt, kCap);
+    for (int i = *ntrans + threadIdx.x; i < n; i += kNT) {
+        const unsigned long long key = t.buf[i];
+        const uint32_t id = (uint32_t)__ldg(ids + (uint32_t)(key & 0xFFFFFFFFull));
+        t.buf[i] = (key & 0xFFFFFFFF00000000ull) | id;
+    }
+    // the compaction that follows starts with a barrier
+}
+
+template <bool DBG>
+__global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams p, const int64_t nitems) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    const int tid = threadIdx.x;
+    const int lane = tid & 31;
+    const int warp = tid >> 5;
+    const int c = tid & (kW - 1);   // subspace of this thread in the table build
+    const int u = tid / kW;         // first entry of this thread (0..63)
+    const int half = lane >> 4;
+    const int ksub = p.ksub;
+
+    // ---- shared-memory carve-up: auxiliary data below the table region ----
+    const uint32_t win = (uint32_t)__cvta_generic_to_shared(smem);
+    if (win + (uint32_t)wide_aux_bytes(p.nprobe, DBG) > kLutWin) {  // uniform: layout does not fit this window offset
+        if (tid == 0) atomicOr(p.status, kFlagLayout);
+        return;
+    }
+    unsigned char* const lut_gen = smem + (kLutWin - win);   // table region as a generic pointer
+    float* const cb_s = reinterpret_cast<float*>(smem + (kCbWin - win));
+    unsigned char* a = smem;
+    unsigned long long* kbuf = reinterpret_cast<unsigned long long*>(a);
+    a += (size_t)kCap * 8;
+    ProbeMeta* meta = reinterpret_cast<ProbeMeta*>(a);
+    a += kMetaCap * sizeof(ProbeMeta);
+    float* qs = reinterpret_cast<float*>(a);
+    float* cent_s = qs + kD;          // [2][128]
+    float* r2 = cent_s + 2 * kD;      // [16]
+    a += kD * 4 + 2 * kD * 4 + 64;
+    unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(a);
+    int* cnt_p = reinterpret_cast<int*>(a + 8);
+    int* ntrans_p = cnt_p + 1;
+    a += 32;
+    int* hist_p = reinterpret_cast<int*>(a);
+    a += kQuickWords * 4;
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(a);                        // DBG only: [2][16][8]
+    long long* vprefix = reinterpret_cast<long long*>(a + 2 * kW * 8 * 4);     // DBG only
+    TopkState t{kbuf, cnt_p, tau_p, hist_p};
+
+    // ---- codebook: entries u, u + 64 in registers; u + 128, u + 192 of every thread in shared
+    //      memory as [entry - 128][half of the 8 dimensions][subspace][4 floats] ----
+    float cbr[2][kDsub];
+#pragma unroll
+    for (int m = 0; m < kNE; ++m) {
+        const int e = u + kEP * m;
+        const float4* src = reinterpret_cast<const float4*>(p.cbt + ((size_t)e * kW + c) * kDsub);
+        const float4 v0 = __ldg(src), v1 = __ldg(src + 1);
+        if (m < 2) {
+            cbr[m][0] = v0.x; cbr[m][1] = v0.y; cbr[m][2] = v0.z; cbr[m][3] = v0.w;
+            cbr[m][4] = v1.x; cbr[m][5] = v1.y; cbr[m][6] = v1.z; cbr[m][7] = v1.w;
+        } else {
+            float4* dst = reinterpret_cast<float4*>(cb_s + (size_t)(e - 128) * (2 * kW * 4));
+            dst[c] = v0;
+            dst[kW + c] = v1;
+        }
+    }
+    // row u, columns c and c + 16; the two half-warps (rows u, u + 1) write the copies in opposite
+    // order so that a warp's 32 stores hit 32 banks
+    const int st_a = u * kRowBytes + (c + (half ? 16 : 0)) * 4;
+    const int st_b = u * kRowBytes + (c + (half ? 0 : 16)) * 4;
+    // column offsets (lane ^ i) * 4 of the 16 steps, four per register
+    uint32_t pk[4];
+#pragma unroll
+    for (int k4 = 0; k4 < 4; ++k4) {
+        uint32_t v = 0;
+#pragma unroll
+        for (int tt = 0; tt < 4; ++tt) v |= (uint32_t)(((lane ^ (4 * k4 + tt)) * 4) & 0xFF) << (8 * tt);
+        pk[k4] = v;
+    }
+
+    // This thread's share of a table (steps B, C + selection): residual of subspace c from the
+    // staged centroid, squared distance to its four entries, kept when within the threshold.
+    auto build = [&](unsigned char* lutb, const float* cs, float thr, float P, uint32_t* hm) {
+        float r[kDsub];
+        {
+            const float4 qa = *reinterpret_cast<const float4*>(qs + c * kDsub);
+            const float4 qb = *reinterpret_cast<const float4*>(qs + c * kDsub + 4);
+            const float4 ca = *reinterpret_cast<const float4*>(cs + c * kDsub);
+            const float4 cb = *reinterpret_cast<const float4*>(cs + c * kDsub + 4);
+            r[0] = __fsub_rn(qa.x, ca.x); r[1] = __fsub_rn(qa.y, ca.y);
+            r[2] = __fsub_rn(qa.z, ca.z); r[3] = __fsub_rn(qa.w, ca.w);
+            r[4] = __fsub_rn(qb.x, cb.x); r[5] = __fsub_rn(qb.y, cb.y);
+            r[6] = __fsub_rn(qb.z, cb.z); r[7] = __fsub_rn(qb.w, cb.w);
+        }
+#pragma unroll
+        for (int m = 0; m < kNE; ++m) {
+            float e8[kDsub];
+            if (m < 2) {
+#pragma unroll
+                for (int j = 0; j < kDsub; ++j) e8[j] = cbr[m < 2 ? m : 0][j];
+            } else {
+                const float4* src = reinterpret_cast<const float4*>(cb_s + (size_t)(u + kEP * (m - 2)) * (2 * kW * 4));
+                const float4 v0 = src[c], v1 = src[kW + c];
+                e8[0] = v0.x; e8[1] = v0.y; e8[2] = v0.z; e8[3] = v0.w;
+                e8[4] = v1.x; e8[5] = v1.y; e8[6] = v1.z; e8[7] = v1.w;
+            }
+            float d2 = 0.0f;
+#pragma unroll
+            for (int j = 0; j < kDsub; ++j) {
+                const float tt = __fsub_rn(r[j], e8[j]);
+                d2 = __fmaf_rn(tt, tt, d2);
+            }
+            const int e = u + kEP * m;
+            const bool hit = e < ksub && (p.dense || d2 <= thr);
+            const float val = hit ? d2 : P;
+            unsigned char* row = lutb + m * (kEP * kRowBytes);
+            *reinterpret_cast<float*>(row + st_a) = val;
+            *reinterpret_cast<float*>(row + st_b) = val;
+            if (DBG && hit) atomicOr(&hm[c * 8 + (e >> 5)], 1u << (e & 31));
+        }
+    };
+    // copies centroid `cl` (128 floats) into cs[0..128): one float4 per thread of one warp
+    auto fetch_cent = [&](int cl, float* cs, int l) { cp_async16(cs + 4 * l, p.cent + (int64_t)cl * kD + 4 * l); };
+
+    topk_quick_init<kNT>(hist_p);  // contains a barrier: the shared half of the codebook is complete too
+
+    for (int64_t item = blockIdx.x; item < nitems; item += gridDim.x) {
+        const int64_t q = item / p.nsplit;
+        const int split = (int)(item % p.nsplit);
+        const int np_item = (p.nprobe - split + p.nsplit - 1) / p.nsplit;  // probes split, split + nsplit, ...
+        __syncthreads();  // the previous item's results have been read out of the candidate buffer
+        if (tid < kW) {
+            float v = 0.0f;
+            if (!p.dense) {
+                const float* rad = p.radius_mode == 1 ? p.radius + q * kW : p.radius;
+                const float r = __fmul_rn(rad[tid], p.scale);
+                v = __fmul_rn(r, r);
+            }
+            r2[tid] = v;
+        } else if (tid >= 32 && tid < 64) {
+            reinterpret_cast<float4*>(qs)[tid - 32] = __ldg(reinterpret_cast<const float4*>(p.queries + q * kD) + (tid - 32));
+        } else if (tid == 64) {
+            *cnt_p = 0;
+            *ntrans_p = 0;
+            *tau_p = kKeyPad;
+        }
+        if (DBG && tid == 96) {
+            long long run = 0;
+            for (int i = 0; i < p.nprobe; ++i) {
+                vprefix[i] = run;
+                const int cl = p.probe_ids[q * p.nprobe + i];
+                if (cl >= 0 && cl < p.nlist) run += p.list_off[cl + 1] - p.list_off[cl];
+            }
+            vprefix[p.nprobe] = run;
+            if (p.visit_count) p.visit_count[q] = run;
+        }
+        float P = 0.0f, thr = 0.0f;
+
+        for (int t0 = 0; t0 < np_item; t0 += kMetaCap) {
+            const int nt = min(kMetaCap, np_item - t0);
+            // ---- stage the metadata of the tile's clusters (the previous tile ended with a barrier) ----
+            if (tid >= 128 && tid < 128 + nt) {
+                const int i = tid - 128;
+                const int pi = split + (t0 + i) * p.nsplit;
+                int cl = p.probe_ids[q * p.nprobe + pi];
+                ProbeMeta m;
+                m.len = 0;
+                m.b0 = 0;
+                m.p0 = 0;
+                m.pad = 0;
+                if (cl < 0 || cl >= p.nlist) {
+                    atomicOr(p.status, kFlagBadList);
+                    cl = 0;
+                } else {
+                    const long long p0 = p.list_off[cl], p1 = p.list_off[cl + 1];
+                    const long long b0 = p.list_blk[cl], b1 = p.list_blk[cl + 1];
+                    const long long len = p1 - p0;
+                    if (len < 0 || p1 > 0x7FFFFFFFll || b1 - b0 != (len + kPointsPerBlock - 1) / kPointsPerBlock) {
+                        atomicOr(p.status, kFlagBadList);
+                    } else {
+                        m.len = (int)len;
+                        m.b0 = b0;
+                        m.p0 = (int)p0;
+                    }
+                }
+                m.cl = cl;
+                meta[i] = m;
+            }
+            if (DBG)
+                for (int i = tid; i < 2 * kW * 8; i += kNT) hitmask[i] = 0;
+            __syncthreads();
+            if (t0 == 0) {
+                if (!p.dense) {
+                    if (p.miss_penalty >= 0.0f) {
+                        P = p.miss_penalty;
+                    } else {
+#pragma unroll
+                        for (int s = 0; s < kW; ++s) P = __fadd_rn(P, r2[s]);
+                    }
+                }
+                thr = r2[c];
+            }
+
+            // ---- prologue: centroids of the tile's first two clusters, table of the first ----
+            if (tid < 32) fetch_cent(meta[0].cl, cent_s, tid);
+            else if (tid < 64 && nt > 1) fetch_cent(meta[1].cl, cent_s + kD, tid - 32);
+            cp_async_wait_all();
+            __syncthreads();
+            build(lut_gen, cent_s, thr, P, hitmask);
+            __syncthreads();
+
+            for (int j = 0; j < nt; ++j) {
+                const ProbeMeta m = meta[j];
+                const int pi = split + (t0 + j) * p.nsplit;
+                const int nblk = (m.len + kPointsPerBlock - 1) / kPointsPerBlock;
+                const uint4* cp = reinterpret_cast<const uint4*>(p.codes_il) + m.b0 * 32 + lane;
+                // the warp's first two code blocks: requested now, needed after the table build
+                int blk = warp;
+                uint4 n0 = make_uint4(0, 0, 0, 0), n1 = make_uint4(0, 0, 0, 0);
+                if (blk < nblk) n0 = __ldg(cp + (int64_t)blk * 32);
+                if (blk + kWarps < nblk) n1 = __ldg(cp + (int64_t)(blk + kWarps) * 32);
+                // the warp's first blocks of the next list: into L2 while this list is scanned
+                if (kPfDist > 0 && j + 1 < nt) {
+                    const ProbeMeta m1 = meta[j + 1];
+                    const int nblk1 = (m1.len + kPointsPerBlock - 1) / kPointsPerBlock;
+                    const uint4* cp1 = reinterpret_cast<const uint4*>(p.codes_il) + m1.b0 * 32 + lane;
+#pragma unroll
+                    for (int i = 0; i < 3; ++i)
+                        if (warp + i * kWarps < nblk1) prefetch_l2(cp1 + (int64_t)(warp + i * kWarps) * 32);
+                }
+                // centroid of cluster j + 2 into the slot that the build of table j read
+                if (tid < 32 && j + 2 < nt) fetch_cent(meta[j + 2].cl, cent_s + (j & 1) * kD, tid);
+
+                if (DBG) {
+                    // masks of cluster j are complete (previous barrier); clear the other buffer
+                    if (p.masks)
+                        for (int i = tid; i < kW * 8; i += kNT)
+                            p.masks[(q * p.nprobe + pi) * kW * 8 + i] = hitmask[(j & 1) * kW * 8 + i];
+                    for (int i = tid; i < kW * 8; i += kNT) hitmask[((j + 1) & 1) * kW * 8 + i] = 0;
+                    __syncthreads();
+                }
+                // ---- this thread's share of the next cluster's table ----
+                if (j + 1 < nt)
+                    build(lut_gen + ((j + 1) & 1) * 128, cent_s + ((j + 1) & 1) * kD, thr, P, hitmask + ((j + 1) & 1) * kW * 8);
+
+                // ---- scan the list of cluster j (step D) ----
+                const uint32_t* hm = hitmask + (j & 1) * kW * 8;
+                while (true) {
+                    const uint32_t tau_hi = (uint32_t)(*tau_p >> 32);
+                    auto scan_blocks = [&](auto table_tag) {
+                        constexpr int TABLE = decltype(table_tag)::value;
+                        while (blk < nblk) {
+                            if (*reinterpret_cast<volatile int*>(cnt_p) >= kSoftLimit) break;
+                            const uint4 cur = n0;
+                            n0 = n1;
+                            if (blk + 2 * kWarps < nblk) n1 = __ldg(cp + (int64_t)(blk + 2 * kWarps) * 32);
+                            if (kPfDist > 0 && blk + kPfDist * kWarps < nblk) prefetch_l2(cp + (int64_t)(blk + kPfDist * kWarps) * 32);
+                            const float acc = gather16<TABLE>(cur, pk);
+                            const int pos = blk * kPointsPerBlock + lane;
+                            if (pos < m.len) {
+                                if (DBG) {
+                                    unsigned long long hs = 0;
+                                    const uint32_t wv[4] = {cur.x, cur.y, cur.z, cur.w};
+#pragma unroll
+                                    for (int i = 0; i < kW; ++i) {
+                                        const uint32_t code = (wv[i >> 2] >> (8 * (i & 3))) & 0xFFu;
+                                        const int s = (lane ^ i) & (kW - 1);
+                                        hs |= (unsigned long long)((hm[s * 8 + (code >> 5)] >> (code & 31)) & 1u) << s;
+                                    }
+                                    const int64_t vi = vprefix[pi] + pos;
+                                    if (vi < p.visit_stride) {
+                                        if (p.visit_hits) p.visit_hits[q * p.visit_stride + vi] = hs;
+                                        if (p.visit_dist) p.visit_dist[q * p.visit_stride + vi] = acc;
+                                        if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[m.p0 + pos];
+                                    }
+                                }
+                                // distance-only test: a tie with the threshold distance is sorted out
+                                // at the next compaction, once the id is known
+                                if (__float_as_uint(acc) <= tau_hi) {
+                                    const int slot = atomicAdd(cnt_p, 1);
+                                    if (slot < kCap) kbuf[slot] = make_key(acc, (uint32_t)(m.p0 + pos));
+                                    else atomicOr(p.status, kFlagOverflow);
+                                }
+                            }
+                            blk += kWarps;
+                        }
+                    };
+                    if (j & 1) scan_blocks(std::integral_constant<int, 1>{});
+                    else scan_blocks(std::integral_constant<int, 0>{});
+                    cp_async_wait_all();
+                    // the barrier that separates cluster j from cluster j + 1 (table j + 1 complete,
+                    // table j free); a set flag means some warp stopped at the soft limit
+                    if (!__syncthreads_or(blk < nblk)) break;
+                    translate_new_keys(t, ntrans_p, p.ids);
+                    topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);
+                    if (tid == 0) *ntrans_p = *cnt_p;  // read again only after later barriers
+                }
+            }
+        }
+
+        // ---- the exact k smallest (distance, id), ascending (paper Sec. 2.1, last paragraph) ----
+        translate_new_keys(t, ntrans_p, p.ids);
+        topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);  // leaves k or a few more keys; starts with a barrier
+        __syncthreads();
+        const int n = min(*cnt_p, kCap);
+        if (p.nsplit == 1) {
+            float* od = p.out_dist + q * p.k;
+            int32_t* oi = p.out_ids + q * p.k;
+            topk_emit_ranked<kNT, CtaGroup>(t, n, p.k, [&](int rank, unsigned long long key) {
+                od[rank] = __uint_as_float((uint32_t)(key >> 32));
+                oi[rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
+            });
+            for (int i = n + tid; i < p.k; i += kNT) {
+                od[i] = __uint_as_float((uint32_t)(kKeyPad >> 32));
+                oi[i] = -1;
+            }
+        } else {
+            unsigned long long* dst = p.partial + (q * p.nsplit + split) * p.k;
+            topk_emit_ranked<kNT, CtaGroup>(t, n, p.k, [&](int rank, unsigned long long key) { dst[rank] = key; });
+            for (int i = n + tid; i < p.k; i += kNT) dst[i] = kKeyPad;
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_scan_wide(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
+                             cudaStream_t st) {
+    (void)nprobe;
+    const size_t smem = (size_t)kCbWin + 65536;  // covers both regions for any window offset
+    int64_t grid = ix->sm_count;
+    if (grid > nitems) grid = nitems;
+    cudaError_t e;
+    if (debug) {
+        auto kern = scan_wide16x8_kernel<true>;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)grid, kNT, smem, st>>>(sp, nitems);
+    } else {
+        auto kern = scan_wide16x8_kernel<false>;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<(unsigned)grid, kNT, smem, st>>>(sp, nitems);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace ivfpq

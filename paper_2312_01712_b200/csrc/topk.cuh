@@ -77,11 +77,11 @@ __device__ inline void bitonic_sort(unsigned long long* buf, int n2) {
 
 // Keeps the k smallest keys of the buffer (unordered) and sets the threshold to an exclusive
 // upper bound of the kept keys.  No-op when at most k keys are buffered.  NT = threads per CTA.
-template <int NT, class G = CtaGroup>
+template <int NT, class G = CtaGroup, int CAP = kTopkCap>
 __device__ inline void topk_select(const TopkState& t, int k) {
-    constexpr int kPerThread = (kTopkCap + NT - 1) / NT;
+    constexpr int kPerThread = (CAP + NT - 1) / NT;
     G::sync();
-    const int n = min(*t.cnt, kTopkCap);
+    const int n = min(*t.cnt, CAP);
     if (n <= k) return;  // uniform over the CTA
     const int tid = G::tid();
     unsigned long long prefix = 0;  // high digits of the k-th smallest key found so far
@@ -208,13 +208,13 @@ __device__ __forceinline__ void topk_quick_init(int* qs) {
 // that boundary.  No-op when at most k keys are buffered.  Falls back to the exact selection when
 // the histogram cannot separate the distances (e.g. all equal).  Must be called by all threads of
 // the group; contains barriers.
-template <int NT, class G = CtaGroup>
+template <int NT, class G = CtaGroup, int CAP = kTopkCap>
 __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
-    constexpr int kPerThread = (kTopkCap + NT - 1) / NT;
+    constexpr int kPerThread = (CAP + NT - 1) / NT;
     constexpr int B = kQuickBins;
     static_assert(NT >= B && NT % 32 == 0, "one bin per thread of the first B threads");
     G::sync();
-    const int n = min(*t.cnt, kTopkCap);
+    const int n = min(*t.cnt, CAP);
     if (n <= k) return;  // uniform over the group
     const int tid = G::tid();
     unsigned* uq = reinterpret_cast<unsigned*>(qs);
@@ -275,7 +275,7 @@ __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
     if (tid < kQuickWords - B) qs[B + tid] = (tid == 0) ? -1 : 0;
     if (kept >= n) {  // uniform: nothing would be dropped
         G::sync();
-        topk_select<NT, G>(t, k);  // uses the same shared words as its histogram
+        topk_select<NT, G, CAP>(t, k);  // uses the same shared words as its histogram
         topk_quick_init<NT, G>(qs);
         return;
     }

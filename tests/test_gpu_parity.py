@@ -128,6 +128,37 @@ def test_stage_dumps_bit_equal(shaped, name):
     assert_visits_parity(g, o, wl.index.nsub)
 
 
+@pytest.mark.parametrize("kernel", ["pers", "wide"])
+def test_16x8_kernels_forced(kernel, monkeypatch):
+    """The 16 x 8 shape has two kernels, chosen by mean list length when the index is loaded;
+    force each of them on the same small index: top-k parity (dense, sparse) and stage dumps."""
+    monkeypatch.setenv("IVFPQ_SCAN_KERNEL", kernel)
+    wl = Workload(small_cfg("c1", n=40_000, ncomp=300, nlist=64, nq=70, chunk=16384, kmeans_iters=4))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        q = dev(wl.queries)
+        for nprobe, k in ((7, 100), (64, 1000), (1, 10)):
+            d, i = lib.ivfpq_search_dense(h, q, nprobe, k)
+            o = oracle.search(wl.index, wl.queries, nprobe, k, dense=True)
+            check_status(h)
+            assert_topk_parity(host(d), host(i), o["dist"], o["ids"])
+            d, i = lib.ivfpq_search_sparse(h, q, nprobe, dev(wl.radius_per_query), k, scale=0.9)
+            o = oracle.search(wl.index, wl.queries, nprobe, k, radius=wl.radius_per_query, scale=0.9)
+            check_status(h)
+            assert_topk_parity(host(d), host(i), o["dist"], o["ids"])
+        nq, nprobe, stride = 16, 5, 8000
+        qs, rad = wl.queries[:nq], wl.radius_per_query[:nq]
+        g = lib.ivfpq_debug_search(h, dev(qs), nprobe, 50, radius=dev(rad), scale=1.1, visit_stride=stride)
+        check_status(h)
+        g = {k2: host(v) for k2, v in g.items()}
+        o = oracle.search(wl.index, qs, nprobe, 50, radius=rad, scale=1.1, dumps=True, visit_stride=stride)
+        assert np.array_equal(g["masks"].view(np.uint32), o["masks"])
+        assert_visits_parity(g, o, wl.index.nsub)
+        assert_topk_parity(g["dist"], g["ids"], o["dist"], o["ids"])
+    finally:
+        lib.ivfpq_index_free(h)
+
+
 @pytest.mark.parametrize("mode", ["per_subspace", "per_query"])
 @pytest.mark.parametrize("scale,penalty", [(1.0, -1.0), (0.5, -1.0), (2.0, 123.5), (0.0, 3.0), (float("inf"), -1.0)])
 def test_sparse_search_matches_oracle(loaded, mode, scale, penalty):
