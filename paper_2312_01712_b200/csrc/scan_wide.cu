@@ -332,11 +332,16 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                 const int pi = split + (t0 + j) * p.nsplit;
                 const int nblk = (m.len + kPointsPerBlock - 1) / kPointsPerBlock;
                 const uint4* cp = reinterpret_cast<const uint4*>(p.codes_il) + m.b0 * 32 + lane;
-                // the warp's first two code blocks: requested now, needed after the table build
-                int blk = warp;
+                // The warp owns blocks warp, warp + 32, ...: `rem` of them are left, `ptr` is this lane's
+                // 16 bytes of the next one, `pos` the position of the lane's point in the list.  The
+                // first two blocks are requested now and needed after the table build.
+                constexpr int kStep = kWarps * 32;   // uint4 elements between two blocks of a warp
+                int rem = nblk > warp ? (nblk - warp + kWarps - 1) / kWarps : 0;
+                const uint4* ptr = cp + warp * 32;
+                int pos = warp * kPointsPerBlock + lane;
                 uint4 n0 = make_uint4(0, 0, 0, 0), n1 = make_uint4(0, 0, 0, 0);
-                if (blk < nblk) n0 = __ldg(cp + (int64_t)blk * 32);
-                if (blk + kWarps < nblk) n1 = __ldg(cp + (int64_t)(blk + kWarps) * 32);
+                if (rem > 0) n0 = __ldg(ptr);
+                if (rem > 1) n1 = __ldg(ptr + kStep);
                 // the warp's first blocks of the next list: into L2 while this list is scanned
                 if (kPfDist > 0 && j + 1 < nt) {
                     const ProbeMeta m1 = meta[j + 1];
@@ -367,14 +372,13 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                     const uint32_t tau_hi = (uint32_t)(*tau_p >> 32);
                     auto scan_blocks = [&](auto table_tag) {
                         constexpr int TABLE = decltype(table_tag)::value;
-                        while (blk < nblk) {
+                        while (rem > 0) {
                             if (*reinterpret_cast<volatile int*>(cnt_p) >= kSoftLimit) break;
                             const uint4 cur = n0;
                             n0 = n1;
-                            if (blk + 2 * kWarps < nblk) n1 = __ldg(cp + (int64_t)(blk + 2 * kWarps) * 32);
-                            if (kPfDist > 0 && blk + kPfDist * kWarps < nblk) prefetch_l2(cp + (int64_t)(blk + kPfDist * kWarps) * 32);
+                            if (rem > 2) n1 = __ldg(ptr + 2 * kStep);
+                            if (kPfDist > 0 && rem > kPfDist) prefetch_l2(ptr + kPfDist * kStep);
                             const float acc = gather16<TABLE>(cur, pk);
-                            const int pos = blk * kPointsPerBlock + lane;
                             if (pos < m.len) {
                                 if (DBG) {
                                     unsigned long long hs = 0;
@@ -400,7 +404,9 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                                     else atomicOr(p.status, kFlagOverflow);
                                 }
                             }
-                            blk += kWarps;
+                            ptr += kStep;
+                            pos += kWarps * kPointsPerBlock;
+                            --rem;
                         }
                     };
                     if (j & 1) scan_blocks(std::integral_constant<int, 1>{});
@@ -408,7 +414,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                     cp_async_wait_all();
                     // the barrier that separates cluster j from cluster j + 1 (table j + 1 complete,
                     // table j free); a set flag means some warp stopped at the soft limit
-                    if (!__syncthreads_or(blk < nblk)) break;
+                    if (!__syncthreads_or(rem > 0)) break;
                     translate_new_keys(t, ntrans_p, p.ids);
                     topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);
                     if (tid == 0) *ntrans_p = *cnt_p;  // read again only after later barriers
