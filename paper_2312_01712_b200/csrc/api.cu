@@ -14,7 +14,8 @@ namespace {
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 struct DerivedLayout {
-    size_t list_off_off, list_blk_off, codes_off, cbt_off, total;
+    size_t list_off_off, list_blk_off, codes_off, cbt_off, cnorm_off, total;
+    int32_t mma;
     int64_t nblocks, max_len;
     int32_t nw, vec16;
     int32_t rot, gw[3], block_bytes;
@@ -53,6 +54,9 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     off = align_up(off + (size_t)nblocks * out->block_bytes, 256);
     out->cbt_off = off;
     if (out->rot) off = align_up(off + (size_t)d->nsub * 256 * d->dsub * 4, 256);
+    out->cnorm_off = off;
+    out->mma = coarse_mma_supported(d->d, d->nlist) ? 1 : 0;
+    if (out->mma) off = align_up(off + coarse_mma_derived_bytes(d->nlist), 256);
     out->total = off > 0 ? off : 256;
     return IVFPQ_OK;
 }
@@ -211,6 +215,7 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     for (int i = 0; i < 3; ++i) ix->gw[i] = dl.rot ? dl.gw[i] : 0;
     ix->block_bytes = dl.block_bytes;
     ix->cbt = reinterpret_cast<const float*>(base + dl.cbt_off);
+    ix->cnorm = dl.mma ? reinterpret_cast<const float*>(base + dl.cnorm_off) : nullptr;
     ix->max_list_len = dl.max_len;
     ix->device = dev;
     ix->sm_count = sms;
@@ -240,6 +245,8 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     if (e == cudaSuccess)
         e = launch_relayout(ix, desc->codes, reinterpret_cast<uint32_t*>(base + dl.codes_off),
                             reinterpret_cast<float*>(base + dl.cbt_off), st);
+    if (e == cudaSuccess && ix->cnorm)
+        e = launch_cnorm(ix->cent, ix->nlist, ix->d, reinterpret_cast<float*>(base + dl.cnorm_off), st);
     if (e != cudaSuccess) {
         delete ix;
         return IVFPQ_ERR_CUDA;

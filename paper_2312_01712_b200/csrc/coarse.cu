@@ -112,8 +112,16 @@ __global__ void __launch_bounds__(256) select_probes_kernel(const float* __restr
 cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,
                           float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
                           int* status, cudaStream_t st, int64_t* launches) {
+    // tensor-core proposal + exact decision when the shape allows it (16-byte aligned rows)
+    const bool mma = ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
+                     (reinterpret_cast<uintptr_t>(ix->cent) & 15) == 0;
     for (int64_t q0 = 0; q0 < nq; q0 += qchunk) {
         const int nqc = (int)((nq - q0 < qchunk) ? (nq - q0) : qchunk);
+        if (mma) {
+            const cudaError_t e = launch_coarse_mma(ix, queries, q0, nqc, nprobe, coarse_tile, probe_ids, probe_d, status, st, launches);
+            if (e == cudaSuccess) continue;
+            if (e != cudaErrorNotSupported) return e;
+        }
         dim3 grid((ix->nlist + TC - 1) / TC, (nqc + TQ - 1) / TQ);
         coarse_dist_kernel<<<grid, 256, 0, st>>>(queries, q0, nqc, ix->cent, ix->nlist, ix->d, coarse_tile);
         select_probes_kernel<<<nqc, 256, 0, st>>>(coarse_tile, ix->nlist, nprobe, probe_ids, probe_d, q0, status);

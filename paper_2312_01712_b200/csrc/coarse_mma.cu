@@ -1,0 +1,482 @@
+// Filtering stage on the 5th-generation tensor cores (paper Sec. 2.1 "Online Search", step A; the
+// GEMM form |c|^2 - 2 q.c + |q|^2 of Sec. 4.3, last paragraph).
+//
+// The tensor cores only *propose*: the nprobe closest clusters are decided by the defining fp32
+// arithmetic (sum over dimensions of fma(t, t, acc), t = q_j - c_j, j ascending), because the probe
+// lists must not depend on how a GEMM rounds.
+//
+//   1. coarse_mma_kernel: approx[q][c] = |c|^2 - 2 q.c for a tile of queries against all centroids.
+//      TMA (cp.async.bulk.tensor, 128-byte swizzle) stages fp32 tiles of queries and centroids in
+//      shared memory as they are in global memory (both are K-major: the dimension runs fastest);
+//      one elected thread issues tcgen05.mma kind::tf32 (128 x 128 x 8 per instruction) into a
+//      double-buffered fp32 accumulator in tensor memory; four warps read the accumulator back
+//      with tcgen05.ld and write the approximate distances.
+//   2. probe_rerank_kernel (one CTA per query): the nprobe-th smallest approximate distance plus
+//      twice a rigorous error bound of the TF32 products gives a cut that no true member of the
+//      answer can exceed; every centroid under the cut is re-evaluated with the defining
+//      arithmetic and the nprobe smallest (distance, cluster id) are returned.  When the cut lets
+//      too many centroids through, the CTA evaluates all of them exactly instead.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out raises the status flag, the roles
+// leave their loops, the tensor memory is released and the kernel returns.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "topk.cuh"
+
+namespace ivfpq {
+
+namespace {
+
+constexpr int kTileM = 128;          // queries per CTA tile (= TMEM lanes)
+constexpr int kTileN = 128;          // centroids per MMA tile (= TMEM columns per accumulator)
+constexpr int kKBlock = 32;          // fp32 elements per 128-byte swizzle row
+constexpr int kTileBytes = kTileM * kKBlock * 4;   // one [128 rows][128 bytes] tile: 16 KB
+constexpr int kStages = 4;           // centroid tiles in flight
+constexpr int kMaxKBlocks = 8;       // dimension <= 256
+constexpr int kMmaThreads = 192;     // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int kTmemCols = 256;       // two accumulators of 128 columns
+constexpr unsigned kSpinLimit = 1u << 22;
+constexpr int kCandCap = kTopkCap;   // centroids that may pass the cut before the exact fallback
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false (and the abort word set) when it ran out or somebody else gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int* status) {
+    for (unsigned i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try(bar, parity)) return true;
+        if (*abort_word) return false;
+    }
+    *abort_word = 1;
+    atomicOr(status, kFlagTimeout);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x 128 x 8, TF32 inputs, fp32 accumulation.
+__device__ __forceinline__ void tc_mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{ .reg .pred p; setp.ne.b32 p, %4, 0;\n"
+        "  tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, {%5, %5, %5, %5}, p; }"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+// 32 lanes x 32 consecutive columns of 32-bit accumulators: thread = lane, v[i] = column i.
+__device__ __forceinline__ void tc_load_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major [rows][128 bytes] tile with 128-byte swizzle: rows
+// are 128 bytes apart, groups of 8 rows 1024 bytes apart; `k_bytes` selects the 32-byte slice of the
+// row that one TF32 instruction (K = 8) consumes.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t tile_addr, int k_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)(((tile_addr + (uint32_t)k_bytes) >> 4) & 0x3FFFu);   // start address
+    d |= (uint64_t)1 << 16;                                              // leading byte offset (16 B; unused here)
+    d |= (uint64_t)(1024 >> 4) << 32;                                    // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                                              // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                                              // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: fp32 accumulator, TF32 A and B, both K-major, N = 128, M = 128.
+constexpr uint32_t kInstrDesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTileN >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+
+struct MmaShared {
+    unsigned long long q_full;
+    unsigned long long full[kStages];
+    unsigned long long empty[kStages];
+    unsigned long long acc_full[2];
+    unsigned long long acc_empty[2];
+    uint32_t tmem_base;
+    int abort_word;
+};
+
+// out[(q - q0) * nlist + c] = cnorm[c] - 2 q.c (TF32 products), q in [q0, q0 + nqc), all c.
+// grid.x: query tiles of 128, grid.y: centroid-tile groups.
+__global__ void __launch_bounds__(kMmaThreads, 1)
+coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c,
+                  const float* __restrict__ cnorm, int nqc, int nlist, int kblocks, float* __restrict__ out,
+                  int* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    // the swizzled tiles need 1024-byte alignment in the shared window
+    const uint32_t dyn_addr = smem_u32(dyn);
+    const uint32_t pad = (1024u - (dyn_addr & 1023u)) & 1023u;
+    unsigned char* base = dyn + pad;
+    const uint32_t q_smem = dyn_addr + pad;                                   // kblocks tiles
+    const uint32_t b_smem = q_smem + (uint32_t)kblocks * kTileBytes;          // kStages tiles
+    MmaShared* sh = reinterpret_cast<MmaShared*>(base + (size_t)(kblocks + kStages) * kTileBytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qt = blockIdx.x;
+    const int ntile = (nlist + kTileN - 1) / kTileN;
+    volatile int* abort_word = &sh->abort_word;
+
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&sh->q_full), 1);
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(smem_u32(&sh->full[i]), 1);
+            mbar_init(smem_u32(&sh->empty[i]), 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(smem_u32(&sh->acc_full[i]), 1);
+            mbar_init(smem_u32(&sh->acc_empty[i]), 4);
+        }
+        sh->abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {  // one warp owns the tensor-memory allocation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            mbar_expect_tx(smem_u32(&sh->q_full), (uint32_t)kblocks * kTileBytes);
+            for (int kb = 0; kb < kblocks; ++kb)
+                tma_load_2d(q_smem + kb * kTileBytes, &map_q, kb * kKBlock, qt * kTileM, smem_u32(&sh->q_full));
+            unsigned it = 0;
+            bool ok = true;
+            for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y) {
+                for (int kb = 0; kb < kblocks && ok; ++kb, ++it) {
+                    const unsigned s = it % kStages;
+                    ok = mbar_wait(smem_u32(&sh->empty[s]), ((it / kStages) & 1) ^ 1, abort_word, status);
+                    if (!ok) break;
+                    mbar_expect_tx(smem_u32(&sh->full[s]), kTileBytes);
+                    tma_load_2d(b_smem + s * kTileBytes, &map_c, kb * kKBlock, ct * kTileN, smem_u32(&sh->full[s]));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            bool ok = mbar_wait(smem_u32(&sh->q_full), 0, abort_word, status);
+            unsigned it = 0, t = 0;
+            for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y, ++t) {
+                const unsigned buf = t & 1;
+                ok = mbar_wait(smem_u32(&sh->acc_empty[buf]), ((t >> 1) & 1) ^ 1, abort_word, status);
+                if (!ok) break;
+                tc_fence_after();
+                for (int kb = 0; kb < kblocks && ok; ++kb, ++it) {
+                    const unsigned s = it % kStages;
+                    ok = mbar_wait(smem_u32(&sh->full[s]), (it / kStages) & 1, abort_word, status);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < kKBlock / 8; ++k)
+                        tc_mma_tf32(tmem + buf * kTileN, smem_desc_sw128(q_smem + kb * kTileBytes, k * 32),
+                                    smem_desc_sw128(b_smem + s * kTileBytes, k * 32), kInstrDesc, (kb | k) != 0 ? 1u : 0u);
+                    tc_commit(smem_u32(&sh->empty[s]));   // the stage is free once these MMAs have read it
+                }
+                if (ok) tc_commit(smem_u32(&sh->acc_full[buf]));
+            }
+        }
+    } else {
+        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. + 31 = query rows of the tile ----
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int q = qt * kTileM + row;
+        unsigned t = 0;
+        bool ok = true;
+        for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y, ++t) {
+            const unsigned buf = t & 1;
+            ok = mbar_wait(smem_u32(&sh->acc_full[buf]), (t >> 1) & 1, abort_word, status);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int cc = 0; cc < kTileN / 32; ++cc) {
+                uint32_t v[32];
+                tc_load_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * kTileN + cc * 32, v);
+                const int c0 = ct * kTileN + cc * 32;
+                if (q < nqc) {
+                    float* dst = out + (size_t)q * nlist + c0;
+                    if (c0 + 32 <= nlist && (nlist & 3) == 0) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            const float4 cn = __ldg(reinterpret_cast<const float4*>(cnorm + c0 + i));
+                            float4 o;
+                            o.x = fmaf(-2.0f, __uint_as_float(v[i + 0]), cn.x);
+                            o.y = fmaf(-2.0f, __uint_as_float(v[i + 1]), cn.y);
+                            o.z = fmaf(-2.0f, __uint_as_float(v[i + 2]), cn.z);
+                            o.w = fmaf(-2.0f, __uint_as_float(v[i + 3]), cn.w);
+                            *reinterpret_cast<float4*>(dst + i) = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (c0 + i < nlist) dst[i] = fmaf(-2.0f, __uint_as_float(v[i]), __ldg(cnorm + c0 + i));
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[buf]));
+        }
+    }
+
+    // ---- teardown: everybody is done with tensor memory before it is released ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// |c|^2 per centroid (fp32) and the largest of them (as ordered uint bits).
+__global__ void __launch_bounds__(256) cnorm_kernel(const float* __restrict__ cent, int nlist, int d,
+                                                    float* __restrict__ cnorm, unsigned* __restrict__ cmax_bits) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= nlist) return;
+    float s = 0.0f;
+    for (int j = 0; j < d; ++j) {
+        const float x = cent[(size_t)c * d + j];
+        s = fmaf(x, x, s);
+    }
+    cnorm[c] = s;
+    atomicMax(cmax_bits, __float_as_uint(s));
+}
+
+// One CTA per query: cut from the approximate distances, exact re-evaluation of everything under
+// the cut, the nprobe smallest (distance, cluster id) ascending.
+__global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restrict__ approx, const float* __restrict__ queries,
+                                                          const float* __restrict__ cent, const unsigned* __restrict__ cmax_bits,
+                                                          int nlist, int d, int nprobe, int64_t q0,
+                                                          int32_t* __restrict__ probe_ids, float* __restrict__ probe_d,
+                                                          int* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    unsigned long long* buf = reinterpret_cast<unsigned long long*>(dyn);                 // [kTopkCap]
+    int* cand = reinterpret_cast<int*>(dyn + (size_t)kTopkCap * 8);                       // [kCandCap]
+    float* qs = reinterpret_cast<float*>(cand + kCandCap);                                // [d]
+    __shared__ int cnt;
+    __shared__ unsigned long long tau;
+    __shared__ int hist[kQuickWords];   // also the exact selection's histogram (kTopkHistInts words)
+    __shared__ float red[8];
+    __shared__ int ncand;
+    static_assert(kQuickWords >= kTopkHistInts, "shared histogram words");
+    TopkState t{buf, &cnt, &tau, hist};
+    const int tid = threadIdx.x;
+    const int64_t q = q0 + blockIdx.x;
+    const float* row = approx + (size_t)blockIdx.x * nlist;
+
+    float part = 0.0f;
+    for (int j = tid; j < d; j += 256) {
+        const float x = queries[q * d + j];
+        qs[j] = x;
+        part = fmaf(x, x, part);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    if ((tid & 31) == 0) red[tid >> 5] = part;
+    if (tid == 0) ncand = 0;
+    for (int i = tid; i < kQuickWords; i += 256) hist[i] = (i == kQuickBins) ? -1 : 0;
+    topk_init(t);  // contains a barrier
+    float qn = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) qn += red[i];
+    const float cmax = __uint_as_float(*cmax_bits);
+    // |approx - exact| <= eps: TF32 keeps 10 mantissa bits of each factor (relative 2^-10 each, 2^-9
+    // per product), summed over the dimensions by Cauchy-Schwarz and doubled by the factor -2; the
+    // second term covers fp32 accumulation and the rounding of the exact side.
+    const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + 3.8e-6f * (qn + cmax);
+
+    // exact squared distance by the defining arithmetic (rows are 16-byte aligned, d % 4 == 0)
+    auto exact = [&](int c) {
+        const float4* cv = reinterpret_cast<const float4*>(cent + (size_t)c * d);
+        float a = 0.0f;
+        for (int j4 = 0; j4 < (d >> 2); ++j4) {
+            const float4 cc = __ldg(cv + j4);
+            const float4 qq = *reinterpret_cast<const float4*>(qs + 4 * j4);
+            float tt;
+            tt = __fsub_rn(qq.x, cc.x); a = __fmaf_rn(tt, tt, a);
+            tt = __fsub_rn(qq.y, cc.y); a = __fmaf_rn(tt, tt, a);
+            tt = __fsub_rn(qq.z, cc.z); a = __fmaf_rn(tt, tt, a);
+            tt = __fsub_rn(qq.w, cc.w); a = __fmaf_rn(tt, tt, a);
+        }
+        return a;
+    };
+
+    bool all_exact = nprobe >= nlist;
+    if (!all_exact) {
+        // ---- a bound at or above the nprobe-th smallest approximate distance: stream the row
+        //      through the buffer, compacting by histogram whenever it could overflow ----
+        for (int base = 0; base < nlist; base += 256) {
+            const int c = base + tid;
+            if (c < nlist) {
+                const unsigned long long key = make_key(fmaxf(row[c] + qn, 0.0f), (uint32_t)c);
+                if (key < tau) {
+                    if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
+                }
+            }
+            __syncthreads();
+            const int filled = cnt;
+            __syncthreads();
+            if (filled + 256 > kTopkCap) topk_quick_compact<256>(t, nprobe, hist);
+        }
+        topk_quick_compact<256>(t, nprobe, hist);   // starts and ends with a barrier
+        const float bound = __uint_as_float((uint32_t)(tau >> 32));   // every kept key is below it; +inf when nothing was dropped
+        const float cut = bound + 2.0f * eps;
+        __syncthreads();
+        // ---- everything under the cut ----
+        for (int c = tid; c < nlist; c += 256) {
+            if (fmaxf(row[c] + qn, 0.0f) <= cut) {
+                const int pos = atomicAdd(&ncand, 1);
+                if (pos < kCandCap) cand[pos] = c;
+            }
+        }
+        __syncthreads();
+        all_exact = ncand > kCandCap;   // uniform
+    }
+    __syncthreads();
+    topk_init(t);
+    if (all_exact) {
+        for (int base = 0; base < nlist; base += 256) {
+            const int c = base + tid;
+            if (c < nlist) {
+                const unsigned long long key = make_key(exact(c), (uint32_t)c);
+                if (key < tau) {
+                    if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
+                }
+            }
+            topk_round_end<256>(t, nprobe, 256);
+        }
+        topk_finalize<256>(t, nprobe);
+        for (int i = tid; i < nprobe; i += 256) {
+            const unsigned long long key = i < cnt ? buf[i] : kKeyPad;
+            probe_ids[q * nprobe + i] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
+            probe_d[q * nprobe + i] = __uint_as_float((uint32_t)(key >> 32));
+        }
+    } else {
+        const int n = ncand;   // nprobe <= n <= kCandCap = buffer size
+        for (int i = tid; i < n; i += 256) {
+            const int c = cand[i];
+            buf[i] = make_key(exact(c), (uint32_t)c);
+        }
+        __syncthreads();
+        topk_emit_ranked<256>(t, n, nprobe, [&](int rank, unsigned long long key) {
+            probe_ids[q * nprobe + rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
+            probe_d[q * nprobe + rank] = __uint_as_float((uint32_t)(key >> 32));
+        });
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess) return nullptr;
+        if (qres != cudaDriverEntryPointSuccess) return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// [rows][d] fp32 row-major, boxes of 128 rows x 32 columns, 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap* map, const float* ptr, int64_t rows, int d) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)d * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)kKBlock, (cuuint32_t)kTileM};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool coarse_mma_supported(int d, int nlist) {
+    return d % 4 == 0 && d >= 4 && (d + kKBlock - 1) / kKBlock <= kMaxKBlocks && nlist >= 1 && encode_tiled_fn() != nullptr;
+}
+
+size_t coarse_mma_derived_bytes(int nlist) { return align_up((size_t)nlist * 4, 256) + 256; }
+
+// Fills cnorm[nlist] and the max word behind it (derived buffer of the index).
+cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st) {
+    unsigned* cmax = reinterpret_cast<unsigned*>(reinterpret_cast<char*>(cnorm) + align_up((size_t)nlist * 4, 256));
+    cudaError_t e = cudaMemsetAsync(cmax, 0, 4, st);
+    if (e != cudaSuccess) return e;
+    cnorm_kernel<<<(nlist + 255) / 256, 256, 0, st>>>(cent, nlist, d, cnorm, cmax);
+    return cudaGetLastError();
+}
+
+// Tensor-core filtering of the queries [q0, q0 + nqc): returns cudaErrorNotSupported when the
+// tensor maps cannot be built (the caller then uses the plain kernels).
+cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe,
+                              float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
+                              int64_t* launches) {
+    alignas(64) CUtensorMap map_q, map_c;
+    if (!make_map(&map_q, queries + q0 * ix->d, nqc, ix->d)) return cudaErrorNotSupported;
+    if (!make_map(&map_c, ix->cent, ix->nlist, ix->d)) return cudaErrorNotSupported;
+    const int kblocks = (ix->d + kKBlock - 1) / kKBlock;
+    const int qtiles = (nqc + kTileM - 1) / kTileM;
+    const int ntile = (ix->nlist + kTileN - 1) / kTileN;
+    int csplit = (2 * ix->sm_count + qtiles - 1) / qtiles;   // about two waves of CTAs
+    if (csplit > ntile) csplit = ntile;
+    if (csplit < 1) csplit = 1;
+    const size_t smem = 1024 + (size_t)(kblocks + kStages) * kTileBytes + sizeof(MmaShared);
+    cudaError_t e = cudaFuncSetAttribute(coarse_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const float* cnorm = ix->cnorm;
+    const unsigned* cmax = reinterpret_cast<const unsigned*>(reinterpret_cast<const char*>(cnorm) + align_up((size_t)ix->nlist * 4, 256));
+    coarse_mma_kernel<<<dim3(qtiles, csplit), kMmaThreads, smem, st>>>(map_q, map_c, cnorm, nqc, ix->nlist, kblocks, tile, status);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const size_t smem2 = (size_t)kTopkCap * 8 + (size_t)kCandCap * 4 + align_up((size_t)ix->d * 4, 16);
+    e = cudaFuncSetAttribute(probe_rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    if (e != cudaSuccess) return e;
+    probe_rerank_kernel<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
+                                                  probe_d, status);
+    *launches += 2;
+    return cudaGetLastError();
+}
+
+}  // namespace ivfpq

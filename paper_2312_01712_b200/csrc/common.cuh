@@ -43,6 +43,7 @@ struct ivfpq_index {
     int32_t gw[3];            // group widths, largest first, 0 = unused
     int32_t block_bytes;      // bytes of one 32-point code block in the rotated layout
     const float* cbt;         // [group][entry 0..255][column][dsub]
+    const float* cnorm;       // [nlist] squared centroid norms + their maximum (tensor-core filtering), or null
     int64_t max_list_len;
     // host state
     int32_t device;
@@ -104,6 +105,13 @@ cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_
 bool rot_group_widths(int nsub, int w[3]);
 int rot_block_bytes(const int w[3]);
 bool rot_supported(int nsub, int dsub);
+// Tensor-core filtering (coarse_mma.cu).
+bool coarse_mma_supported(int d, int nlist);
+size_t coarse_mma_derived_bytes(int nlist);
+cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st);
+cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe,
+                              float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
+                              int64_t* launches);
 cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,
                           float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
                           int* status, cudaStream_t st, int64_t* launches);

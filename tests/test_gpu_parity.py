@@ -69,6 +69,30 @@ def test_probe_lists_bit_equal(loaded, name, nprobe):
     assert np.array_equal(host(pd).view(np.uint32), opd.view(np.uint32))
 
 
+def test_probe_lists_tensor_core_shapes():
+    """Filtering through the tensor-core proposal + exact decision on shapes that exercise the
+    tile edges: d = 200 (seven 32-float K blocks, the last one zero-filled beyond the row),
+    nlist = 300 (three centroid tiles, the last one partly outside), 300 queries (three query tiles)."""
+    wl = Workload(small_cfg("c4", n=30_000, ncomp=300, nlist=300, nq=300, chunk=16384, kmeans_iters=3))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        q = dev(wl.queries)
+        for nprobe in (1, 9, 64, 300):
+            pid, pd = lib.ivfpq_debug_probes(h, q, nprobe)
+            opid, opd = oracle.coarse(wl.index, wl.queries, nprobe)
+            check_status(h)
+            assert np.array_equal(host(pid), opid)
+            assert np.array_equal(host(pd).view(np.uint32), opd.view(np.uint32))
+        # rows that are not 16-byte aligned take the plain kernels: same answer
+        q_off = torch.empty(wl.queries.size + 1, dtype=torch.float32, device="cuda")[1:].view(wl.queries.shape)
+        q_off.copy_(q)
+        pid2, pd2 = lib.ivfpq_debug_probes(h, q_off, 9)
+        pid, pd = lib.ivfpq_debug_probes(h, q, 9)
+        assert torch.equal(pid, pid2) and torch.equal(pd.view(torch.int32), pd2.view(torch.int32))
+    finally:
+        lib.ivfpq_index_free(h)
+
+
 def test_probe_all_lists(loaded):
     wl, h = loaded["small"]
     pid, pd = lib.ivfpq_debug_probes(h, dev(wl.queries), wl.index.nlist)
