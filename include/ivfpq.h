@@ -101,7 +101,7 @@ typedef struct {
 size_t ivfpq_search_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k);
 
 /* Conventional (dense) IVFPQ search: every codebook entry is selected.
- * queries dev [nq][d]; out_dist dev [nq][k] ascending; out_ids dev [nq][k]; ties are ordered by
+ * queries dev [nq][d], 16-byte aligned; out_dist dev [nq][k] ascending; out_ids dev [nq][k]; ties are ordered by
  * ascending id; when fewer than k points were visited the tail is (+inf, -1). */
 int ivfpq_search_dense(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
                        int32_t k, float* out_dist, int32_t* out_ids, void* workspace,

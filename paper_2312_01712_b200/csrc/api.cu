@@ -80,6 +80,7 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
         if (isnan(a.scale) || isnan(a.miss_penalty)) return IVFPQ_ERR_INVALID_ARGUMENT;
     }
     if (!aligned(a.queries, 4) || !aligned(workspace, 256)) return IVFPQ_ERR_WORKSPACE;
+    if (!probes_only && !aligned(a.queries, 16)) return IVFPQ_ERR_INVALID_ARGUMENT;  // the scan kernels load rows as float4
     const WorkspaceLayout wl = plan_workspace(ix, a.nq, a.nprobe, a.k);
     if (workspace_bytes < wl.total) return IVFPQ_ERR_WORKSPACE;
 

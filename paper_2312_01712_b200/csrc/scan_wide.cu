@@ -50,7 +50,7 @@ constexpr int kCap = 4096;        // candidate buffer slots
 constexpr int kSoftLimit = 2048;  // compaction is requested once this many candidates are buffered
 constexpr int kMetaCap = 128;     // clusters whose metadata is staged at a time
 constexpr int kPfDist = 3;         // blocks (per warp) that the L2 prefetch runs ahead of the scan
-static_assert(kSoftLimit + kNT <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
+static_assert(kSoftLimit + 2 * kNT <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
 
 struct ProbeMeta {
     long long b0;   // first 32-point code block of the list
@@ -348,7 +348,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                     const int nblk1 = (m1.len + kPointsPerBlock - 1) / kPointsPerBlock;
                     const uint4* cp1 = reinterpret_cast<const uint4*>(p.codes_il) + m1.b0 * 32 + lane;
 #pragma unroll
-                    for (int i = 0; i < 3; ++i)
+                    for (int i = 0; i < 4; ++i)
                         if (warp + i * kWarps < nblk1) prefetch_l2(cp1 + (int64_t)(warp + i * kWarps) * 32);
                 }
                 // centroid of cluster j + 2 into the slot that the build of table j read
@@ -370,16 +370,14 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                 const uint32_t* hm = hitmask + (j & 1) * kW * 8;
                 while (true) {
                     const uint32_t tau_hi = (uint32_t)(*tau_p >> 32);
+                    bool stop = false;   // a candidate of this lane landed at or beyond the soft limit
+                    bool halt = false;   // ... of this warp, as seen at the end of a round
                     auto scan_blocks = [&](auto table_tag) {
                         constexpr int TABLE = decltype(table_tag)::value;
-                        while (rem > 0) {
-                            if (*reinterpret_cast<volatile int*>(cnt_p) >= kSoftLimit) break;
-                            const uint4 cur = n0;
-                            n0 = n1;
-                            if (rem > 2) n1 = __ldg(ptr + 2 * kStep);
-                            if (kPfDist > 0 && rem > kPfDist) prefetch_l2(ptr + kPfDist * kStep);
+                        // one block: 16 look-ups per lane, stage dumps, candidate test
+                        auto one = [&](const uint4 cur, const int bpos) {
                             const float acc = gather16<TABLE>(cur, pk);
-                            if (pos < m.len) {
+                            if (bpos < m.len) {
                                 if (DBG) {
                                     unsigned long long hs = 0;
                                     const uint32_t wv[4] = {cur.x, cur.y, cur.z, cur.w};
@@ -389,32 +387,55 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                                         const int s = (lane ^ i) & (kW - 1);
                                         hs |= (unsigned long long)((hm[s * 8 + (code >> 5)] >> (code & 31)) & 1u) << s;
                                     }
-                                    const int64_t vi = vprefix[pi] + pos;
+                                    const int64_t vi = vprefix[pi] + bpos;
                                     if (vi < p.visit_stride) {
                                         if (p.visit_hits) p.visit_hits[q * p.visit_stride + vi] = hs;
                                         if (p.visit_dist) p.visit_dist[q * p.visit_stride + vi] = acc;
-                                        if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[m.p0 + pos];
+                                        if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[m.p0 + bpos];
                                     }
                                 }
                                 // distance-only test: a tie with the threshold distance is sorted out
                                 // at the next compaction, once the id is known
                                 if (__float_as_uint(acc) <= tau_hi) {
                                     const int slot = atomicAdd(cnt_p, 1);
-                                    if (slot < kCap) kbuf[slot] = make_key(acc, (uint32_t)(m.p0 + pos));
+                                    if (slot < kCap) kbuf[slot] = make_key(acc, (uint32_t)(m.p0 + bpos));
                                     else atomicOr(p.status, kFlagOverflow);
+                                    stop |= slot >= kSoftLimit;
                                 }
                             }
-                            ptr += kStep;
-                            pos += kWarps * kPointsPerBlock;
-                            --rem;
+                        };
+                        // Two blocks per round; each code register is refilled right after its block
+                        // has been consumed (no copies).  The fill level of the candidate buffer is
+                        // only looked at by lanes that push: a warp leaves the loop at the end of a
+                        // round in which one of its candidates landed beyond the soft limit, which
+                        // bounds the overshoot by 64 candidates per warp.
+                        while (rem >= 2 && !halt) {
+                            one(n0, pos);
+                            if (rem > 2) n0 = __ldg(ptr + 2 * kStep);
+                            one(n1, pos + kWarps * kPointsPerBlock);
+                            if (rem > 3) n1 = __ldg(ptr + 3 * kStep);
+                            if (kPfDist > 0) {
+                                if (rem > kPfDist + 1) prefetch_l2(ptr + (kPfDist + 1) * kStep);
+                                if (rem > kPfDist + 2) prefetch_l2(ptr + (kPfDist + 2) * kStep);
+                            }
+                            ptr += 2 * kStep;
+                            pos += 2 * kWarps * kPointsPerBlock;
+                            rem -= 2;
+                            halt = __any_sync(0xFFFFFFFFu, stop);
+                        }
+                        if (rem == 1 && !halt) {
+                            one(n0, pos);
+                            rem = 0;
+                            halt = __any_sync(0xFFFFFFFFu, stop);
                         }
                     };
                     if (j & 1) scan_blocks(std::integral_constant<int, 1>{});
                     else scan_blocks(std::integral_constant<int, 0>{});
                     cp_async_wait_all();
                     // the barrier that separates cluster j from cluster j + 1 (table j + 1 complete,
-                    // table j free); a set flag means some warp stopped at the soft limit
-                    if (!__syncthreads_or(rem > 0)) break;
+                    // table j free); a set flag means some warp saw the soft limit (it may have
+                    // finished its blocks all the same: the buffer is compacted before the next list)
+                    if (!__syncthreads_or(rem > 0 || halt)) break;
                     translate_new_keys(t, ntrans_p, p.ids);
                     topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);
                     if (tid == 0) *ntrans_p = *cnt_p;  // read again only after later barriers
