@@ -23,8 +23,8 @@
 //     code blocks of a list are requested before the table build and arrive during it;
 //   * candidates go to the CTA's candidate buffer as (distance, position in the id array): the
 //     id itself is read only when the buffer is compacted, for all new candidates at once, so
-//     the scan loop never waits for that load.  A warp checks a soft fill limit before every block
-//     and the CTA compacts only when that limit was hit, with one histogram pass over the
+//     the scan loop never waits for that load.  Only lanes that push look at the fill level; the
+//     CTA compacts when a candidate landed beyond a soft limit, with one histogram pass over the
 //     distances (topk.cuh); the final k are ranked by counting and written straight to the output.
 #include "common.cuh"
 #include "scan_common.cuh"
@@ -42,9 +42,10 @@ constexpr int kEP = kNT / kW;     // entries per pass (32)
 constexpr int kNE = 256 / kEP;    // entries per thread (8)
 constexpr int kRowBytes = 256;    // one table row
 constexpr int kLutBytes = 256 * kRowBytes;  // one table: 64 KB
-constexpr int kSoftLimit = 1536;  // compaction is requested once this many candidates are buffered
+constexpr int kCap = 4096;        // candidate buffer slots
+constexpr int kSoftLimit = 2048;  // compaction is requested once a candidate lands beyond this many
 constexpr int kMetaCap = 128;     // clusters whose metadata is staged at a time
-static_assert(kSoftLimit + kNT <= kTopkCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
+static_assert(kSoftLimit + 2 * kNT <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
 
 struct ProbeMeta {
     long long b0;   // first 32-point code block of the list
@@ -55,7 +56,7 @@ struct ProbeMeta {
 
 // Auxiliary shared memory (everything except the two tables), in bytes.
 __host__ __device__ inline int pers_aux_bytes(int nprobe, bool dbg) {
-    int b = kTopkCap * 8;                 // candidate keys
+    int b = kCap * 8;                     // candidate keys
     b += kMetaCap * (int)sizeof(ProbeMeta);
     b += kW * kDsub * 4;                  // query
     b += 64 * 4;                          // squared thresholds (padded)
@@ -111,7 +112,7 @@ __device__ __forceinline__ float gather16(const uint4 cur, uint32_t bsel) {
 // barrier that follows the last push; the first *ntrans keys already hold ids.
 __device__ __forceinline__ void translate_new_keys(const TopkState& t, const int* ntrans,
                                                    const int32_t* __restrict__ ids) {
-    const int n = min(*t.cnt, kTopkCap);
+    const int n = min(*t.cnt, kCap);
     for (int i = *ntrans + threadIdx.x; i < n; i += kNT) {
         const unsigned long long key = t.buf[i];
         const uint32_t id = (uint32_t)__ldg(ids + (uint32_t)(key & 0xFFFFFFFFull));
@@ -140,7 +141,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
     const int aux_bytes = pers_aux_bytes(p.nprobe, DBG);
     unsigned char* const aux = (pad >= (uint32_t)aux_bytes) ? smem : smem + pad + 2 * kLutBytes;
     unsigned long long* kbuf = reinterpret_cast<unsigned long long*>(aux);
-    ProbeMeta* meta = reinterpret_cast<ProbeMeta*>(aux + (size_t)kTopkCap * 8);
+    ProbeMeta* meta = reinterpret_cast<ProbeMeta*>(aux + (size_t)kCap * 8);
     float* qs = reinterpret_cast<float*>(meta + kMetaCap);
     float* r2 = qs + d;
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + 64);
@@ -291,11 +292,16 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
                 const int pi = split + (t0 + j) * p.nsplit;
                 const int nblk = (m.len + kPointsPerBlock - 1) / kPointsPerBlock;
                 const uint4* cp = reinterpret_cast<const uint4*>(p.codes_il) + m.b0 * 32 + lane;
-                // the warp's first two code blocks: requested now, needed after the table build
-                int blk = warp;
+                // The warp owns blocks warp, warp + 16, ...: `rem` of them are left, `ptr` is this lane's
+                // 16 bytes of the next one, `pos` the position of the lane's point in the list.  The
+                // first two blocks are requested now and needed after the table build.
+                constexpr int kStep = kWarps * 32;   // uint4 elements between two blocks of a warp
+                int rem = nblk > warp ? (nblk - warp + kWarps - 1) / kWarps : 0;
+                const uint4* ptr = cp + warp * 32;
+                int pos = warp * kPointsPerBlock + lane;
                 uint4 n0 = make_uint4(0, 0, 0, 0), n1 = make_uint4(0, 0, 0, 0);
-                if (blk < nblk) n0 = __ldg(cp + (int64_t)blk * 32);
-                if (blk + kWarps < nblk) n1 = __ldg(cp + (int64_t)(blk + kWarps) * 32);
+                if (rem > 0) n0 = __ldg(ptr);
+                if (rem > 1) n1 = __ldg(ptr + kStep);
 
                 if (DBG) {
                     // masks of cluster j are complete (previous barrier); clear the other buffer
@@ -318,14 +324,12 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
                 const uint32_t* hm = hitmask + (j & 1) * kW * 8;
                 while (true) {
                     const uint32_t tau_hi = (uint32_t)(*tau_p >> 32);
-                    while (blk < nblk) {
-                        if (*reinterpret_cast<volatile int*>(cnt_p) >= kSoftLimit) break;
-                        const uint4 cur = n0;
-                        n0 = n1;
-                        if (blk + 2 * kWarps < nblk) n1 = __ldg(cp + (int64_t)(blk + 2 * kWarps) * 32);
+                    bool stop = false;   // a candidate of this lane landed at or beyond the soft limit
+                    bool halt = false;   // ... of this warp, as seen at the end of a round
+                    // one block: 16 look-ups per lane, stage dumps, candidate test
+                    auto one = [&](const uint4 cur, const int bpos) {
                         const float acc = gather16(cur, bsel);
-                        const int pos = blk * kPointsPerBlock + lane;
-                        if (pos < m.len) {
+                        if (bpos < m.len) {
                             if (DBG) {
                                 unsigned long long hs = 0;
                                 const uint32_t wv[4] = {cur.x, cur.y, cur.z, cur.w};
@@ -335,27 +339,49 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
                                     const int s = (lane + i) & (kW - 1);
                                     hs |= (unsigned long long)((hm[s * 8 + (code >> 5)] >> (code & 31)) & 1u) << s;
                                 }
-                                const int64_t vi = vprefix[pi] + pos;
+                                const int64_t vi = vprefix[pi] + bpos;
                                 if (vi < p.visit_stride) {
                                     if (p.visit_hits) p.visit_hits[q * p.visit_stride + vi] = hs;
                                     if (p.visit_dist) p.visit_dist[q * p.visit_stride + vi] = acc;
-                                    if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[m.p0 + pos];
+                                    if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[m.p0 + bpos];
                                 }
                             }
                             // distance-only test: a tie with the threshold distance is sorted out
                             // at the next compaction, once the id is known
                             if (__float_as_uint(acc) <= tau_hi) {
-                                if (!topk_push(t, make_key(acc, (uint32_t)(m.p0 + pos))))
-                                    atomicOr(p.status, kFlagOverflow);
+                                const int slot = atomicAdd(cnt_p, 1);
+                                if (slot < kCap) kbuf[slot] = make_key(acc, (uint32_t)(m.p0 + bpos));
+                                else atomicOr(p.status, kFlagOverflow);
+                                stop |= slot >= kSoftLimit;
                             }
                         }
-                        blk += kWarps;
+                    };
+                    // Two blocks per round; each code register is refilled right after its block has
+                    // been consumed (no copies).  The fill level of the candidate buffer is only
+                    // looked at by lanes that push: a warp leaves the loop at the end of a round in
+                    // which one of its candidates landed beyond the soft limit, which bounds the
+                    // overshoot by 64 candidates per warp.
+                    while (rem >= 2 && !halt) {
+                        one(n0, pos);
+                        if (rem > 2) n0 = __ldg(ptr + 2 * kStep);
+                        one(n1, pos + kWarps * kPointsPerBlock);
+                        if (rem > 3) n1 = __ldg(ptr + 3 * kStep);
+                        ptr += 2 * kStep;
+                        pos += 2 * kWarps * kPointsPerBlock;
+                        rem -= 2;
+                        halt = __any_sync(0xFFFFFFFFu, stop);
+                    }
+                    if (rem == 1 && !halt) {
+                        one(n0, pos);
+                        rem = 0;
+                        halt = __any_sync(0xFFFFFFFFu, stop);
                     }
                     // the barrier that separates cluster j from cluster j + 1 (table j + 1 complete,
-                    // table j free); a set flag means some warp stopped at the soft limit
-                    if (!__syncthreads_or(blk < nblk)) break;
+                    // table j free); a set flag means some warp saw the soft limit (it may have
+                    // finished its blocks all the same: the buffer is compacted before the next list)
+                    if (!__syncthreads_or(rem > 0 || halt)) break;
                     translate_new_keys(t, ntrans_p, p.ids);
-                    topk_quick_compact<kNT>(t, p.k, hist_p);
+                    topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);
                     if (tid == 0) *ntrans_p = *cnt_p;  // read again only after later barriers
                 }
             }
@@ -363,9 +389,9 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
 
         // ---- the exact k smallest (distance, id), ascending (paper Sec. 2.1, last paragraph) ----
         translate_new_keys(t, ntrans_p, p.ids);
-        topk_quick_compact<kNT>(t, p.k, hist_p);   // leaves k or a few more keys; starts with a barrier
+        topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);   // leaves k or a few more keys; starts with a barrier
         __syncthreads();
-        const int n = min(*cnt_p, kTopkCap);
+        const int n = min(*cnt_p, kCap);
         if (p.nsplit == 1) {
             float* od = p.out_dist + q * p.k;
             int32_t* oi = p.out_ids + q * p.k;
