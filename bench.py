@@ -111,13 +111,29 @@ class ClockSampler:
 # workload
 # --------------------------------------------------------------------------------------------
 
-def build_workload(name: str, device: str, nq: int | None, query_seed_offset: int = 0):
-    """Index + queries + exact neighbours + calibrated radii for one of the synthetic configs."""
+def rank_config(name: str, nq: int | None, rank: int):
+    """The workload of one rank: the index recipe is the same on every rank (replicated index), the
+    query batch is drawn from a rank-specific seed (queries are sharded, no exchange)."""
     cfg = CONFIGS[name]
     if nq is not None:
         cfg = cfg.scaled(nq=nq)
-    if query_seed_offset:
-        cfg = cfg.scaled(query_seed=cfg.query_seed + query_seed_offset)
+    if rank:
+        cfg = cfg.scaled(query_seed=cfg.query_seed + rank)
+    return cfg
+
+
+def max_over_ranks(total_ms: float, dist, device) -> float:
+    """Device time of the slowest rank (all ranks search concurrently)."""
+    if dist is None:
+        return total_ms
+    t = torch.tensor([total_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def build_workload(name: str, device: str, nq: int | None, query_seed_offset: int = 0):
+    """Index + queries + exact neighbours + calibrated radii for one of the synthetic configs."""
+    cfg = rank_config(name, nq, query_seed_offset)
     t0 = time.time()
     spec = G.make_mixture(cfg, device)
     q = G.queries(cfg, spec)
@@ -241,12 +257,7 @@ def run_cuda(args):
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
-        total_ms = sum(a.elapsed_time(b) for a, b in evs)
-        if dist is not None:
-            t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total_ms = float(t.item())
-        return total_ms
+        return max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), dist, dev)
 
     sampler = ClockSampler(local_rank)
     stages = []
