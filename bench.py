@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one scan-kernel launch, from the ncu captures
 # summarised under profiles/ (bytes per launch of the benchmark's workload; None = not captured).
-SCAN_DRAM_TRAFFIC_BYTES = {}
+SCAN_DRAM_TRAFFIC_BYTES = {"c2": 26.6e6, "c5": 72.4e9}
 
 
 def log(*a):
@@ -322,7 +322,8 @@ def run_cuda(args):
         "roofline": {"bound": "hbm", "kernel": scan_kernel_name(index) + " (selective LUT + list scan + top-k)",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": f"of {peak_src}", "algorithmic_bytes_per_launch": int(scan_bytes),
-                     "visits_per_launch": int(visits), "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload)},
+                     "visits_per_launch": int(visits),
+                     "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload) if (args.nq is None and args.nprobe == 0) else None},
         "gather_roofline": {"bound": "shared-memory gathers", "achieved": gather_rate, "peak": gather_peak,
                             "unit": "Ggather/s", "frac": gather_rate / gather_peak,
                             "peak_source": f"{props.multi_processor_count} SMs x 32 lanes x {clk:.0f} MHz"},

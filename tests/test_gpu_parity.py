@@ -183,6 +183,31 @@ def test_16x8_kernels_forced(kernel, monkeypatch):
         lib.ivfpq_index_free(h)
 
 
+@pytest.mark.parametrize("kernel", ["pers", "wide"])
+def test_16x8_many_probes_and_splits(kernel, monkeypatch):
+    """More probed clusters than the kernels stage at a time (128), alone and split over several
+    CTAs per query, on an index with short and empty lists."""
+    monkeypatch.setenv("IVFPQ_SCAN_KERNEL", kernel)
+    wl = Workload(small_cfg("c1", n=20_000, ncomp=200, nlist=300, nq=24, chunk=16384, kmeans_iters=3))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        q = dev(wl.queries)
+        for nsplit in (1, 3):
+            lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_NSPLIT, nsplit)
+            for nprobe, k in ((200, 100), (300, 1000), (129, 7)):
+                d, i = lib.ivfpq_search_sparse(h, q, nprobe, dev(wl.radius), k, scale=1.0)
+                check_status(h)
+                o = oracle.search(wl.index, wl.queries, nprobe, k, radius=wl.radius, scale=1.0)
+                assert_topk_parity(host(d), host(i), o["dist"], o["ids"])
+        lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_NSPLIT, 0)
+        d, i = lib.ivfpq_search_dense(h, q, 256, 1024)
+        check_status(h)
+        o = oracle.search(wl.index, wl.queries, 256, 1024, dense=True)
+        assert_topk_parity(host(d), host(i), o["dist"], o["ids"])
+    finally:
+        lib.ivfpq_index_free(h)
+
+
 @pytest.mark.parametrize("mode", ["per_subspace", "per_query"])
 @pytest.mark.parametrize("scale,penalty", [(1.0, -1.0), (0.5, -1.0), (2.0, 123.5), (0.0, 3.0), (float("inf"), -1.0)])
 def test_sparse_search_matches_oracle(loaded, mode, scale, penalty):
