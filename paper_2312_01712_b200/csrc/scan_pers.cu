@@ -26,16 +26,14 @@
 //     the scan loop never waits for that load.  Only lanes that push look at the fill level; the
 //     CTA compacts when a candidate landed beyond a soft limit, with one histogram pass over the
 //     distances (topk.cuh); the final k are ranked by counting and written straight to the output.
-#include "common.cuh"
-#include "scan_common.cuh"
-#include "topk.cuh"
+#include "scan16x8.cuh"
 
 namespace ivfpq {
 
 namespace {
 
-constexpr int kW = 16;            // subspaces
-constexpr int kDsub = 8;
+using namespace pq16x8;
+
 constexpr int kNT = 512;          // threads per CTA
 constexpr int kWarps = kNT / 32;
 constexpr int kEP = kNT / kW;     // entries per pass (32)
@@ -44,15 +42,8 @@ constexpr int kRowBytes = 256;    // one table row
 constexpr int kLutBytes = 256 * kRowBytes;  // one table: 64 KB
 constexpr int kCap = 4096;        // candidate buffer slots
 constexpr int kSoftLimit = 2048;  // compaction is requested once a candidate lands beyond this many
-constexpr int kMetaCap = 128;     // clusters whose metadata is staged at a time
 static_assert(kSoftLimit + 2 * kNT <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
 
-struct ProbeMeta {
-    long long b0;   // first 32-point code block of the list
-    long long p0;   // first point of the list (index into ids)
-    int len;        // points in the list (0 when the cluster id or its tables were invalid)
-    int cl;         // cluster id, clamped into range
-};
 
 // Auxiliary shared memory (everything except the two tables), in bytes.
 __host__ __device__ inline int pers_aux_bytes(int nprobe, bool dbg) {
@@ -107,20 +98,6 @@ __device__ __forceinline__ float gather16(const uint4 cur, uint32_t bsel) {
     return a0 + a1;
 }
 
-// The keys pushed since the last compaction carry the position of the point in the id array;
-// replace it by the id (equal distances are ordered by id).  Called by all threads after a
-// barrier that follows the last push; the first *ntrans keys already hold ids.
-__device__ __forceinline__ void translate_new_keys(const TopkState& t, const int* ntrans,
-                                                   const int32_t* __restrict__ ids) {
-    const int n = min(*t.cnt, kCap);
-    for (int i = *ntrans + threadIdx.x; i < n; i += kNT) {
-        const unsigned long long key = t.buf[i];
-        const uint32_t id = (uint32_t)__ldg(ids + (uint32_t)(key & 0xFFFFFFFFull));
-        t.buf[i] = (key & 0xFFFFFFFF00000000ull) | id;
-    }
-    // the compaction that follows starts with a barrier
-}
-
 template <bool DBG>
 __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams p, const int64_t nitems) {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -131,7 +108,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
     const int u = tid / kW;         // first entry of this thread
     const int half = lane >> 4;
     const int ksub = p.ksub;
-    constexpr int d = kW * kDsub;
+    constexpr int d = kD;
 
     // ---- shared-memory carve-up ----
     const uint32_t win = (uint32_t)__cvta_generic_to_shared(smem);
@@ -211,67 +188,20 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
         const int np_item = (p.nprobe - split + p.nsplit - 1) / p.nsplit;  // probes split, split + nsplit, ...
         __syncthreads();  // the previous item's results have been read out of the candidate buffer
         if (tid < kW) {
-            float v = 0.0f;
-            if (!p.dense) {
-                const float* rad = p.radius_mode == 1 ? p.radius + q * kW : p.radius;
-                const float r = __fmul_rn(rad[tid], p.scale);
-                v = __fmul_rn(r, r);
-            }
-            r2[tid] = v;
+            r2[tid] = squared_threshold(p, q, tid);
         } else if (tid >= 32 && tid < 64) {
             reinterpret_cast<float4*>(qs)[tid - 32] = __ldg(reinterpret_cast<const float4*>(p.queries + q * d) + (tid - 32));
         }
-        if (DBG && tid == 0) {
-            long long run = 0;
-            for (int i = 0; i < p.nprobe; ++i) {
-                vprefix[i] = run;
-                const int cl = p.probe_ids[q * p.nprobe + i];
-                if (cl >= 0 && cl < p.nlist) run += p.list_off[cl + 1] - p.list_off[cl];
-            }
-            vprefix[p.nprobe] = run;
-            if (p.visit_count) p.visit_count[q] = run;
-        }
+        if (DBG && tid == 64) fill_visit_prefix(p, q, vprefix);
         if (tid == 0) *ntrans_p = 0;
         topk_init(t);  // contains a barrier
-        float P = 0.0f;
-        if (!p.dense) {
-            if (p.miss_penalty >= 0.0f) {
-                P = p.miss_penalty;
-            } else {
-#pragma unroll
-                for (int s = 0; s < kW; ++s) P = __fadd_rn(P, r2[s]);
-            }
-        }
+        const float P = miss_constant(p, r2);
         const float thr = r2[c];
 
         for (int t0 = 0; t0 < np_item; t0 += kMetaCap) {
             const int nt = min(kMetaCap, np_item - t0);
             // ---- stage the metadata of the tile's clusters (the previous tile ended with a barrier) ----
-            if (tid < nt) {
-                const int pi = split + (t0 + tid) * p.nsplit;
-                int cl = p.probe_ids[q * p.nprobe + pi];
-                ProbeMeta m;
-                m.len = 0;
-                m.b0 = 0;
-                m.p0 = 0;
-                if (cl < 0 || cl >= p.nlist) {
-                    atomicOr(p.status, kFlagBadList);
-                    cl = 0;
-                } else {
-                    const long long p0 = p.list_off[cl], p1 = p.list_off[cl + 1];
-                    const long long b0 = p.list_blk[cl], b1 = p.list_blk[cl + 1];
-                    const long long len = p1 - p0;
-                    if (len < 0 || len > 0x7FFFFFFFll || b1 - b0 != (len + kPointsPerBlock - 1) / kPointsPerBlock) {
-                        atomicOr(p.status, kFlagBadList);
-                    } else {
-                        m.len = (int)len;
-                        m.b0 = b0;
-                        m.p0 = p0;
-                    }
-                }
-                m.cl = cl;
-                meta[tid] = m;
-            }
+            if (tid < nt) meta[tid] = load_probe_meta(p, q, split + (t0 + tid) * p.nsplit);
             if (DBG)
                 for (int i = tid; i < 2 * kW * 8; i += kNT) hitmask[i] = 0;
             __syncthreads();
@@ -380,34 +310,12 @@ __global__ void __launch_bounds__(kNT, 1) scan_pers16x8_kernel(const ScanParams 
                     // table j free); a set flag means some warp saw the soft limit (it may have
                     // finished its blocks all the same: the buffer is compacted before the next list)
                     if (!__syncthreads_or(rem > 0 || halt)) break;
-                    translate_new_keys(t, ntrans_p, p.ids);
-                    topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);
-                    if (tid == 0) *ntrans_p = *cnt_p;  // read again only after later barriers
+                    compact_candidates<kNT, kCap>(t, ntrans_p, hist_p, p.k, p.ids);
                 }
             }
         }
 
-        // ---- the exact k smallest (distance, id), ascending (paper Sec. 2.1, last paragraph) ----
-        translate_new_keys(t, ntrans_p, p.ids);
-        topk_quick_compact<kNT, CtaGroup, kCap>(t, p.k, hist_p);   // leaves k or a few more keys; starts with a barrier
-        __syncthreads();
-        const int n = min(*cnt_p, kCap);
-        if (p.nsplit == 1) {
-            float* od = p.out_dist + q * p.k;
-            int32_t* oi = p.out_ids + q * p.k;
-            topk_emit_ranked<kNT, CtaGroup>(t, n, p.k, [&](int rank, unsigned long long key) {
-                od[rank] = __uint_as_float((uint32_t)(key >> 32));
-                oi[rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
-            });
-            for (int i = n + tid; i < p.k; i += kNT) {
-                od[i] = __uint_as_float((uint32_t)(kKeyPad >> 32));
-                oi[i] = -1;
-            }
-        } else {
-            unsigned long long* dst = p.partial + (q * p.nsplit + split) * p.k;
-            topk_emit_ranked<kNT, CtaGroup>(t, n, p.k, [&](int rank, unsigned long long key) { dst[rank] = key; });
-            for (int i = n + tid; i < p.k; i += kNT) dst[i] = kKeyPad;
-        }
+        emit_topk<kNT, kCap>(p, t, ntrans_p, hist_p, q, split);
     }
 }
 
