@@ -169,8 +169,8 @@ def scan_kernel_name(index) -> str:
     """Name of the kernel the library picks for this index (same rule as ivfpq_index_load)."""
     if (index.nsub, index.dsub) == (16, 8):
         forced = os.environ.get("IVFPQ_SCAN_KERNEL")
-        wide = forced == "wide" or (forced != "pers" and index.ntotal // index.nlist >= 2048)
-        return "scan_wide16x8_kernel" if wide else "scan_pers16x8_kernel"
+        wide = forced == "warps32" or (forced != "warps16" and index.ntotal // index.nlist >= 2048)
+        return "scan16x8_kernel<1024>" if wide else "scan16x8_kernel<512>"
     return "scan_rot_kernel"
 
 

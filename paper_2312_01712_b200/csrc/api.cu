@@ -204,14 +204,14 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->nblocks = dl.nblocks;
     ix->rot = dl.rot;
     {
-        // 16 x 8 shape: short lists are served best by the 16-warp kernel with the whole codebook
-        // in registers (its table build is the cheaper one), long lists by the 32-warp kernel (its
-        // list scan hides more latency).  IVFPQ_SCAN_KERNEL=pers|wide overrides the choice at load.
+        // 16 x 8 shape: short lists are served best by the 16-warp instance of the persistent kernel
+        // (whole codebook in registers, cheaper table build), long lists by the 32-warp instance (its
+        // list scan hides more latency).  IVFPQ_SCAN_KERNEL=warps16|warps32 overrides the choice at load.
         const int64_t mean_len = desc->nlist > 0 ? desc->ntotal / desc->nlist : 0;
-        ix->pers_kind = mean_len >= 2048 ? 3 : 1;
+        ix->pers_warps = mean_len >= 2048 ? 32 : 16;
         const char* kind = getenv("IVFPQ_SCAN_KERNEL");
-        if (kind && strcmp(kind, "pers") == 0) ix->pers_kind = 1;
-        if (kind && strcmp(kind, "wide") == 0) ix->pers_kind = 3;
+        if (kind && strcmp(kind, "warps16") == 0) ix->pers_warps = 16;
+        if (kind && strcmp(kind, "warps32") == 0) ix->pers_warps = 32;
     }
     for (int i = 0; i < 3; ++i) ix->gw[i] = dl.rot ? dl.gw[i] : 0;
     ix->block_bytes = dl.block_bytes;

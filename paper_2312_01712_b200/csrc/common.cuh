@@ -38,7 +38,7 @@ struct ivfpq_index {
     int64_t nblocks;          // total 32-point blocks
     // rotated layout (scan_rot.cu): subspace groups of power-of-two width, codes stored per lane in
     // the lane's own visiting order, codebook copied entry-major per group
-    int32_t pers_kind;        // 16 x 8 shape: 1 = scan_pers.cu (additive rotation), 3 = scan_wide.cu (xor rotation)
+    int32_t pers_warps;       // 16 x 8 shape: warps per CTA of the persistent kernel (16: short lists, 32: long lists)
     int32_t rot;              // 1: rotated layout in use
     int32_t gw[3];            // group widths, largest first, 0 = unused
     int32_t block_bytes;      // bytes of one 32-point code block in the rotated layout
@@ -57,7 +57,7 @@ struct ivfpq_index {
 
 namespace ivfpq {
 
-// Shape served by the persistent kernel (scan_pers.cu); its code layout is the additive rotation.
+// Shape served by the persistent kernels (scan16x8.cu).
 inline bool pers_shape(const ivfpq_index* ix) { return ix->rot && ix->nsub == 16 && ix->dsub == 8; }
 
 struct SearchArgs {

@@ -54,14 +54,13 @@ __host__ __device__ inline int rot_lane_bytes(int w) { return w >= 16 ? w : (w =
 
 // Rotated layout (see scan_rot.cu): a 32-point block is a sequence of per-group chunks; in the
 // chunk of a group of width w the lane at position `lane` stores, as byte i (i < w), the code of
-// subspace s0 + ((lane ^ i) & (w-1)), or of subspace s0 + ((lane + i) & (w-1)) when `additive` is
-// set (the order the persistent 16 x 8 kernel visits them in).  Lanes are interleaved at the
-// granularity of the vector the scan loads: 16 bytes (w >= 16), 8 bytes (w == 8) or 4 bytes (w <= 4).
+// subspace s0 + ((lane ^ i) & (w-1)).  Lanes are interleaved at the granularity of the vector the
+// scan loads: 16 bytes (w >= 16), 8 bytes (w == 8) or 4 bytes (w <= 4).
 __global__ void __launch_bounds__(256) relayout_rot_kernel(const uint8_t* __restrict__ codes,
                                                            const int64_t* __restrict__ list_off,
                                                            const int64_t* __restrict__ list_blk, int nsub,
                                                            int w0, int w1, int w2, int block_bytes,
-                                                           int additive, unsigned char* __restrict__ dst) {
+                                                           unsigned char* __restrict__ dst) {
     const int list = blockIdx.x;
     const int64_t p0 = list_off[list];
     const int64_t len = list_off[list + 1] - p0;
@@ -82,7 +81,7 @@ __global__ void __launch_bounds__(256) relayout_rot_kernel(const uint8_t* __rest
             const int vec = lb >= 16 ? 16 : lb;  // bytes per lane per vector
             for (int i2 = 0; i2 < lb; ++i2) {
                 unsigned char v = 0;
-                if (i2 < w && pos < len) v = src[s0 + ((additive ? lane + i2 : lane ^ i2) & (w - 1))];
+                if (i2 < w && pos < len) v = src[s0 + ((lane ^ i2) & (w - 1))];
                 // vector number i2 / vec, lanes interleaved per vector
                 blk[chunk + (i2 / vec) * 32 * vec + lane * vec + (i2 % vec)] = v;
             }
@@ -122,7 +121,6 @@ cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_
         if (ix->nblocks > 0)
             relayout_rot_kernel<<<ix->nlist, 256, 0, st>>>(codes, ix->list_off, ix->list_blk, ix->nsub, ix->gw[0],
                                                            ix->gw[1], ix->gw[2], ix->block_bytes,
-                                                           (pers_shape(ix) && ix->pers_kind == 1) ? 1 : 0,
                                                            reinterpret_cast<unsigned char*>(codes_il));
         relayout_cbt_kernel<<<64, 256, 0, st>>>(ix->cb, ix->nsub, ix->dsub, ix->ksub, ix->gw[0], ix->gw[1],
                                                 ix->gw[2], cbt);

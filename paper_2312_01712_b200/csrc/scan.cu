@@ -336,10 +336,8 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     const size_t smem = scan_smem_bytes(ix->nw, ix->d, a.nprobe, a.debug);
     const int64_t grid = a.nq * sp.nsplit;
     cudaError_t e;
-    if (pers_shape(ix) && ix->pers_kind == 3)
-        e = launch_scan_wide(ix, sp, grid, a.debug, a.nprobe, st);
-    else if (pers_shape(ix))
-        e = launch_scan_pers(ix, sp, grid, a.debug, a.nprobe, st);
+    if (pers_shape(ix))
+        e = launch_scan16x8(ix, sp, grid, a.debug, a.nprobe, st);
     else if (ix->rot)
         e = launch_scan_rot(ix, sp, grid, a.debug, a.nprobe, st);
     else

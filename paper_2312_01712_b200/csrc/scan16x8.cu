@@ -1,15 +1,16 @@
 // Persistent fused selective-LUT / list-scan / top-k kernel for the 16 x 8 product quantizer (16
-// subspaces of 8 dimensions, 256 entries), 32 warps per SM.  Same computation as scan.cu (paper
-// Sec. 2.1 steps B-D with the selection of Sec. 3.1 / Algorithm 2 and the miss constant of
-// Sec. 4.3).
+// subspaces of 8 dimensions, 256 entries), the shape of the SIFT-like workloads.  Same computation
+// as scan.cu (paper Sec. 2.1 steps B-D with the selection of Sec. 3.1 / Algorithm 2 and the miss
+// constant of Sec. 4.3).  One CTA per SM loops over (query, probe slice) items.
 //
-//   * One CTA of 1024 threads per SM (64 registers per thread): eight warps per scheduler hide the
-//     latencies of the table gathers and of the code loads that four warps could not.
-//   * The 128 KB codebook stays on chip for the lifetime of the kernel, half in registers and half
-//     in shared memory: thread t owns subspace c = t & 15 and the entries u, u + 64, u + 128,
-//     u + 192 with u = t / 16; the first two live in its registers, the other two are read from
-//     shared memory (two 16-byte loads per entry, conflict-free).  Building a table reads nothing
-//     from global memory but the probed centroid (512 B, copied ahead with cp.async).
+//   * Two instances, chosen when the index is loaded.  16 warps (128 registers per thread): the
+//     whole 128 KB codebook lives in registers - thread t owns subspace c = t & 15 and the entries
+//     u, u + 32, ... with u = t / 16 - which makes the table build cheapest: for short lists,
+//     where the build weighs as much as the scan.  32 warps (64 registers): two entries of a
+//     thread in registers, two in shared memory (two 16-byte loads per entry, conflict-free);
+//     eight warps per scheduler hide the latency of code blocks that stream from HBM: for long
+//     lists.  Either way building a table reads nothing from global memory but the probed centroid
+//     (512 B, copied two clusters ahead with cp.async).
 //   * Table layout: 256 rows (entries) of 256 bytes; a row holds two tables side by side, 32
 //     columns each; column x holds the value of subspace x & 15 (two copies).  Lane l looks up, at
 //     step i, column l ^ i: the 32 lanes of a warp touch 32 different banks whatever the codes
@@ -19,13 +20,14 @@
 //     is the immediate of the load: three instructions per look-up.
 //   * Two tables: while the warps scan the list of cluster j they have already built their share of
 //     the table of cluster j + 1; one barrier per cluster separates the phases.
-//   * Code blocks: two per warp in registers, requested before the table build; further ahead the
-//     warp only asks for the lines to be brought into L2 (prefetch.global.L2, three blocks ahead
-//     and the first blocks of the next list), which keeps enough bytes in flight for lists that
-//     stream from HBM without spending registers.
-//   * Candidates go to the CTA's candidate buffer as (distance, position in the id array); ids are
-//     read when the buffer is compacted (one histogram pass, topk.cuh); the final k are ranked by
-//     counting and written straight to the output.
+//   * Code blocks: two per warp in registers, requested before the table build, refilled in
+//     two-block rounds without register copies; the 32-warp instance also asks for the lines
+//     further ahead to be brought into L2 (prefetch.global.L2, three blocks ahead and the first
+//     blocks of the next list), which keeps enough bytes in flight without spending registers.
+//   * Candidates go to the CTA's candidate buffer as (distance, position in the id array); only
+//     lanes that push look at its fill level; ids are read when the buffer is compacted (one
+//     histogram pass, topk.cuh); the final k are ranked by counting and written straight to the
+//     output.
 #include <type_traits>
 
 #include "scan16x8.cuh"
@@ -36,21 +38,27 @@ namespace {
 
 using namespace pq16x8;
 
-constexpr int kNT = 1024;         // threads per CTA
-constexpr int kWarps = kNT / 32;
-constexpr int kEP = kNT / kW;     // entries per pass (64)
-constexpr int kNE = 256 / kEP;    // entries per thread (4): 0, 1 in registers, 2, 3 in shared memory
+// NT = threads per CTA: 1024 (entries u, u + 64 of a thread in registers, u + 128, u + 192 in shared
+// memory) or 512 (all eight entries of a thread in registers, no shared codebook).
+template <int NT>
+struct Shape {
+    static constexpr int kWarps = NT / 32;
+    static constexpr int kEP = NT / kW;                   // entries per pass
+    static constexpr int kNE = 256 / kEP;                 // entries per thread
+    static constexpr int kRegEntries = NT == 1024 ? 2 : kNE;
+    static_assert(NT == 512 || NT == 1024, "thread counts this kernel is written for");
+};
 constexpr int kRowBytes = 256;    // one table row (two tables side by side)
 constexpr uint32_t kLutWin = 0x10000;   // shared-window address of the table region (64 KB)
 constexpr uint32_t kCbWin = 0x20000;    // shared-window address of the shared half of the codebook (64 KB)
 constexpr int kCap = 4096;        // candidate buffer slots
 constexpr int kSoftLimit = 2048;  // compaction is requested once this many candidates are buffered
 constexpr int kPfDist = 3;         // blocks (per warp) that the L2 prefetch runs ahead of the scan
-static_assert(kSoftLimit + 2 * kNT <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
+static_assert(kSoftLimit + 2 * 1024 <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
 
 
 // Auxiliary shared memory in front of the table region, in bytes.
-__host__ __device__ inline int wide_aux_bytes(int nprobe, bool dbg) {
+__host__ __device__ inline int scan16x8_aux_bytes(int nprobe, bool dbg) {
     int b = kCap * 8;                         // candidate keys
     b += kMetaCap * (int)sizeof(ProbeMeta);
     b += kD * 4 + 2 * kD * 4 + 64;            // query, two centroids, squared thresholds
@@ -94,8 +102,14 @@ __device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[
     return a0 + a1;
 }
 
-template <bool DBG>
-__global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams p, const int64_t nitems) {
+template <int NT, bool DBG>
+__global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, const int64_t nitems) {
+    constexpr int kNT = NT;
+    constexpr int kWarps = Shape<NT>::kWarps;
+    constexpr int kEP = Shape<NT>::kEP;
+    constexpr int kNE = Shape<NT>::kNE;
+    constexpr int kRegEntries = Shape<NT>::kRegEntries;
+    constexpr int kPf = NT == 1024 ? kPfDist : 0;   // the 16-warp instance serves short, L2-resident lists
     extern __shared__ __align__(16) unsigned char smem[];
     const int tid = threadIdx.x;
     const int lane = tid & 31;
@@ -107,7 +121,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
 
     // ---- shared-memory carve-up: auxiliary data below the table region ----
     const uint32_t win = (uint32_t)__cvta_generic_to_shared(smem);
-    if (win + (uint32_t)wide_aux_bytes(p.nprobe, DBG) > kLutWin) {  // uniform: layout does not fit this window offset
+    if (win + (uint32_t)scan16x8_aux_bytes(p.nprobe, DBG) > kLutWin) {  // uniform: layout does not fit this window offset
         if (tid == 0) atomicOr(p.status, kFlagLayout);
         return;
     }
@@ -132,19 +146,21 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
     long long* vprefix = reinterpret_cast<long long*>(a + 2 * kW * 8 * 4);     // DBG only
     TopkState t{kbuf, cnt_p, tau_p, hist_p};
 
-    // ---- codebook: entries u, u + 64 in registers; u + 128, u + 192 of every thread in shared
-    //      memory as [entry - 128][half of the 8 dimensions][subspace][4 floats] ----
-    float cbr[2][kDsub];
+    // ---- codebook: the first kRegEntries entries of a thread in registers, the others (32 warps
+    //      only: entries 128..255) in shared memory as [entry - 128][half of the 8 dimensions]
+    //      [subspace][4 floats] ----
+    float cbr[kRegEntries][kDsub];
 #pragma unroll
     for (int m = 0; m < kNE; ++m) {
         const int e = u + kEP * m;
         const float4* src = reinterpret_cast<const float4*>(p.cbt + ((size_t)e * kW + c) * kDsub);
         const float4 v0 = __ldg(src), v1 = __ldg(src + 1);
-        if (m < 2) {
-            cbr[m][0] = v0.x; cbr[m][1] = v0.y; cbr[m][2] = v0.z; cbr[m][3] = v0.w;
-            cbr[m][4] = v1.x; cbr[m][5] = v1.y; cbr[m][6] = v1.z; cbr[m][7] = v1.w;
+        if (m < kRegEntries) {
+            float* dst = cbr[m < kRegEntries ? m : 0];
+            dst[0] = v0.x; dst[1] = v0.y; dst[2] = v0.z; dst[3] = v0.w;
+            dst[4] = v1.x; dst[5] = v1.y; dst[6] = v1.z; dst[7] = v1.w;
         } else {
-            float4* dst = reinterpret_cast<float4*>(cb_s + (size_t)(e - 128) * (2 * kW * 4));
+            float4* dst = reinterpret_cast<float4*>(cb_s + (size_t)(e - kRegEntries * kEP) * (2 * kW * 4));
             dst[c] = v0;
             dst[kW + c] = v1;
         }
@@ -180,11 +196,11 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
 #pragma unroll
         for (int m = 0; m < kNE; ++m) {
             float e8[kDsub];
-            if (m < 2) {
+            if (m < kRegEntries) {
 #pragma unroll
-                for (int j = 0; j < kDsub; ++j) e8[j] = cbr[m < 2 ? m : 0][j];
+                for (int j = 0; j < kDsub; ++j) e8[j] = cbr[m < kRegEntries ? m : 0][j];
             } else {
-                const float4* src = reinterpret_cast<const float4*>(cb_s + (size_t)(u + kEP * (m - 2)) * (2 * kW * 4));
+                const float4* src = reinterpret_cast<const float4*>(cb_s + (size_t)(u + kEP * (m - kRegEntries)) * (2 * kW * 4));
                 const float4 v0 = src[c], v1 = src[kW + c];
                 e8[0] = v0.x; e8[1] = v0.y; e8[2] = v0.z; e8[3] = v0.w;
                 e8[4] = v1.x; e8[5] = v1.y; e8[6] = v1.z; e8[7] = v1.w;
@@ -262,7 +278,7 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                 if (rem > 0) n0 = __ldg(ptr);
                 if (rem > 1) n1 = __ldg(ptr + kStep);
                 // the warp's first blocks of the next list: into L2 while this list is scanned
-                if (kPfDist > 0 && j + 1 < nt) {
+                if (kPf > 0 && j + 1 < nt) {
                     const ProbeMeta m1 = meta[j + 1];
                     const int nblk1 = (m1.len + kPointsPerBlock - 1) / kPointsPerBlock;
                     const uint4* cp1 = reinterpret_cast<const uint4*>(p.codes_il) + m1.b0 * 32 + lane;
@@ -333,9 +349,9 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
                             if (rem > 2) n0 = __ldg(ptr + 2 * kStep);
                             one(n1, pos + kWarps * kPointsPerBlock);
                             if (rem > 3) n1 = __ldg(ptr + 3 * kStep);
-                            if (kPfDist > 0) {
-                                if (rem > kPfDist + 1) prefetch_l2(ptr + (kPfDist + 1) * kStep);
-                                if (rem > kPfDist + 2) prefetch_l2(ptr + (kPfDist + 2) * kStep);
+                            if (kPf > 0) {
+                                if (rem > kPf + 1) prefetch_l2(ptr + (kPf + 1) * kStep);
+                                if (rem > kPf + 2) prefetch_l2(ptr + (kPf + 2) * kStep);
                             }
                             ptr += 2 * kStep;
                             pos += 2 * kWarps * kPointsPerBlock;
@@ -364,27 +380,33 @@ __global__ void __launch_bounds__(kNT, 1) scan_wide16x8_kernel(const ScanParams 
     }
 }
 
-}  // namespace
-
-cudaError_t launch_scan_wide(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
-                             cudaStream_t st) {
-    (void)nprobe;
-    const size_t smem = (size_t)kCbWin + 65536;  // covers both regions for any window offset
-    int64_t grid = ix->sm_count;
-    if (grid > nitems) grid = nitems;
+template <int NT>
+cudaError_t launch_nt(const ScanParams& sp, int64_t grid, int64_t nitems, bool debug, cudaStream_t st) {
+    // covers the table region (and the shared codebook of the 32-warp kernel) for any window offset
+    const size_t smem = NT == 1024 ? (size_t)kCbWin + 65536 : (size_t)kCbWin;
     cudaError_t e;
     if (debug) {
-        auto kern = scan_wide16x8_kernel<true>;
+        auto kern = scan16x8_kernel<NT, true>;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kern<<<(unsigned)grid, kNT, smem, st>>>(sp, nitems);
+        kern<<<(unsigned)grid, NT, smem, st>>>(sp, nitems);
     } else {
-        auto kern = scan_wide16x8_kernel<false>;
+        auto kern = scan16x8_kernel<NT, false>;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kern<<<(unsigned)grid, kNT, smem, st>>>(sp, nitems);
+        kern<<<(unsigned)grid, NT, smem, st>>>(sp, nitems);
     }
     return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_scan16x8(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
+                             cudaStream_t st) {
+    (void)nprobe;
+    int64_t grid = ix->sm_count;
+    if (grid > nitems) grid = nitems;
+    return ix->pers_warps == 16 ? launch_nt<512>(sp, grid, nitems, debug, st) : launch_nt<1024>(sp, grid, nitems, debug, st);
 }
 
 }  // namespace ivfpq

@@ -1,6 +1,6 @@
-// Pieces shared by the two persistent kernels of the 16 x 8 product quantizer (scan_pers.cu,
-// scan_wide.cu): list metadata staging, the per-query thresholds, the candidate buffer protocol
-// (position keys, compaction, ranked output) and the small PTX helpers.
+// Supporting pieces of the persistent kernel of the 16 x 8 product quantizer (scan16x8.cu): list
+// metadata staging, the per-query thresholds, the candidate buffer protocol (position keys,
+// compaction, ranked output) and the small PTX helpers.
 #pragma once
 
 #include "common.cuh"

@@ -43,12 +43,8 @@ struct ScanParams {
 cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, bool debug,
                             int nprobe, cudaStream_t st);
 
-// Persistent register-resident-codebook scan for the 16 x 8 quantizer (scan_pers.cu).
-cudaError_t launch_scan_pers(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
-                             cudaStream_t st);
-
-// 32-warp persistent scan for the 16 x 8 quantizer, codebook half in registers, half in shared memory (scan_wide.cu).
-cudaError_t launch_scan_wide(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
+// Persistent scan for the 16 x 8 quantizer, 16 or 32 warps per SM (scan16x8.cu).
+cudaError_t launch_scan16x8(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
                              cudaStream_t st);
 
 }  // namespace ivfpq

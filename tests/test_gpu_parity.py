@@ -152,7 +152,7 @@ def test_stage_dumps_bit_equal(shaped, name):
     assert_visits_parity(g, o, wl.index.nsub)
 
 
-@pytest.mark.parametrize("kernel", ["pers", "wide"])
+@pytest.mark.parametrize("kernel", ["warps16", "warps32"])
 def test_16x8_kernels_forced(kernel, monkeypatch):
     """The 16 x 8 shape has two kernels, chosen by mean list length when the index is loaded;
     force each of them on the same small index: top-k parity (dense, sparse) and stage dumps."""
@@ -183,7 +183,7 @@ def test_16x8_kernels_forced(kernel, monkeypatch):
         lib.ivfpq_index_free(h)
 
 
-@pytest.mark.parametrize("kernel", ["pers", "wide"])
+@pytest.mark.parametrize("kernel", ["warps16", "warps32"])
 def test_16x8_many_probes_and_splits(kernel, monkeypatch):
     """More probed clusters than the kernels stage at a time (128), alone and split over several
     CTAs per query, on an index with short and empty lists."""
