@@ -304,7 +304,11 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                 // ---- scan the list of cluster j (step D) ----
                 const uint32_t* hm = hitmask + (j & 1) * kW * 8;
                 while (true) {
-                    const uint32_t tau_hi = (uint32_t)(*tau_p >> 32);
+                    const unsigned long long tau = *tau_p;
+                    const uint32_t tau_hi = (uint32_t)(tau >> 32), tau_lo = (uint32_t)tau;
+                    // one compare in the common case: distances below tau_cut are candidates; a tie with the
+                    // threshold distance (only possible when the threshold carries an id) is then decided by id
+                    const uint32_t tau_cut = tau_hi + (tau_lo != 0 ? 1u : 0u);
                     bool stop = false;   // a candidate of this lane landed at or beyond the soft limit
                     bool halt = false;   // ... of this warp, as seen at the end of a round
                     auto scan_blocks = [&](auto table_tag) {
@@ -329,9 +333,11 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                                         if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[m.p0 + bpos];
                                     }
                                 }
-                                // distance-only test: a tie with the threshold distance is sorted out
-                                // at the next compaction, once the id is known
-                                if (__float_as_uint(acc) <= tau_hi) {
+                                // key < threshold, key = (distance, id).  The id is read only for a tie with
+                                // the threshold distance (many points can share a distance: every point
+                                // that missed in all subspaces has 16 P)
+                                const uint32_t ab = __float_as_uint(acc);
+                                if (ab < tau_cut && (ab != tau_hi || (uint32_t)__ldg(p.ids + m.p0 + bpos) < tau_lo)) {
                                     const int slot = atomicAdd(cnt_p, 1);
                                     if (slot < kCap) kbuf[slot] = make_key(acc, (uint32_t)(m.p0 + bpos));
                                     else atomicOr(p.status, kFlagOverflow);
@@ -371,7 +377,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                     // table j free); a set flag means some warp saw the soft limit (it may have
                     // finished its blocks all the same: the buffer is compacted before the next list)
                     if (!__syncthreads_or(rem > 0 || halt)) break;
-                    compact_candidates<kNT, kCap>(t, ntrans_p, hist_p, p.k, p.ids);
+                    compact_candidates<kNT, kCap>(t, ntrans_p, hist_p, p.k, p.ids, kSoftLimit / 2);   // between lists any cut that frees half the buffer will do
                 }
             }
         }

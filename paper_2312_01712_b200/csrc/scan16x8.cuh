@@ -95,16 +95,17 @@ __device__ inline void fill_visit_prefix(const ScanParams& p, int64_t q, long lo
 // since the last compaction are translated to (distance, id) - equal distances are ordered by id -
 // right before the buffer is compacted; the first *ntrans keys already hold ids.  All threads of
 // the CTA call these after a barrier that follows the last push.
+// `keep_max`: the compaction refines its cut until at most that many keys survive (when it can).
 template <int NT, int CAP>
 __device__ __forceinline__ void compact_candidates(const TopkState& t, int* ntrans, int* qs, int k,
-                                                   const int32_t* __restrict__ ids) {
+                                                   const int32_t* __restrict__ ids, int keep_max) {
     const int n = min(*t.cnt, CAP);
     for (int i = *ntrans + threadIdx.x; i < n; i += NT) {
         const unsigned long long key = t.buf[i];
         const uint32_t id = (uint32_t)__ldg(ids + (uint32_t)(key & 0xFFFFFFFFull));
         t.buf[i] = (key & 0xFFFFFFFF00000000ull) | id;
     }
-    topk_quick_compact<NT, CtaGroup, CAP>(t, k, qs);   // starts and ends with a barrier
+    topk_quick_compact<NT, CtaGroup, CAP, true>(t, k, qs, keep_max);   // starts and ends with a barrier
     if (threadIdx.x == 0) *ntrans = *t.cnt;            // read again only after later barriers
 }
 
@@ -114,7 +115,7 @@ __device__ __forceinline__ void compact_candidates(const TopkState& t, int* ntra
 template <int NT, int CAP>
 __device__ __forceinline__ void emit_topk(const ScanParams& p, const TopkState& t, int* ntrans, int* qs, int64_t q,
                                           int split) {
-    compact_candidates<NT, CAP>(t, ntrans, qs, p.k, p.ids);   // leaves k or a few more keys
+    compact_candidates<NT, CAP>(t, ntrans, qs, p.k, p.ids, p.k + 64);   // leaves k or a few more keys
     __syncthreads();
     const int n = min(*t.cnt, CAP);
     const int tid = threadIdx.x;

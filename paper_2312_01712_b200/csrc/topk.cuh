@@ -205,11 +205,14 @@ __device__ __forceinline__ void topk_quick_init(int* qs) {
 }
 
 // Keeps the keys below a bin boundary chosen so that at least k survive; sets the threshold to
-// that boundary.  No-op when at most k keys are buffered.  Falls back to the exact selection when
-// the histogram cannot separate the distances (e.g. all equal).  Must be called by all threads of
-// the group; contains barriers.
-template <int NT, class G = CtaGroup, int CAP = kTopkCap>
-__device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
+// that boundary.  No-op when at most k keys are buffered.  With REFINE, while more than `keep_max`
+// keys would survive because the boundary bin is crowded (distances bunched together, as the banded
+// distances of the sparsity-aware search are, or many keys sharing one distance), that bin is split
+// again: by finer distance bits, then by the low word of the key.
+// Falls back to the exact selection when the histogram cannot separate the distances (e.g. all
+// equal).  Must be called by all threads of the group; contains barriers.
+template <int NT, class G = CtaGroup, int CAP = kTopkCap, bool REFINE = false>
+__device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs, int keep_max = 0) {
     constexpr int kPerThread = (CAP + NT - 1) / NT;
     constexpr int B = kQuickBins;
     static_assert(NT >= B && NT % 32 == 0, "one bin per thread of the first B threads");
@@ -242,45 +245,120 @@ __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs) {
     const unsigned range = hi - lo;
     int shift = 0;  // smallest shift with (range >> shift) < B
     if (range >= (unsigned)B) shift = (32 - __clz(range)) - (31 - __clz(B));
+
+    // One histogram pass over the keys that `binof` maps to a bin in [0, B): returns the bin that
+    // holds the key of rank `need` among them, the inclusive count up to that bin and the bin's own
+    // count.  Leaves the shared words in their between-calls state again.
+    int bin = 0, incl_total = 0, bin_count = 0;
+    auto hist_pass = [&](auto binof, int need) {
 #pragma unroll
-    for (int j = 0; j < kPerThread; ++j) {
-        const int i = tid + j * NT;
-        if (i < n) atomicAdd(&qs[((unsigned)(mine[j] >> 32) - lo) >> shift], 1);
-    }
-    G::sync();
-    // inclusive prefix sum over the bins, one bin per thread of the first B threads
-    const int v = tid < B ? qs[tid] : 0;
-    int incl = v;
+        for (int j = 0; j < kPerThread; ++j) {
+            const int i = tid + j * NT;
+            const int b = i < n ? binof(mine[j]) : -1;
+            if (b >= 0) atomicAdd(&qs[b], 1);
+        }
+        G::sync();
+        const int v = tid < B ? qs[tid] : 0;
+        int incl = v;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int x = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if ((tid & 31) >= o) incl += x;
-    }
-    if (tid < B && (tid & 31) == 31) qs[B + 4 + (tid >> 5)] = incl;
-    G::sync();
-    if (tid < B) {
-        int before = 0;
-        for (int w = 0; w < (tid >> 5); ++w) before += qs[B + 4 + w];
-        incl += before;
-        if (incl - v < k && k <= incl) {  // exactly one thread: its bin holds the k-th smallest distance
-            qs[B + 2] = tid;
-            qs[B + 3] = incl;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int x = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if ((tid & 31) >= o) incl += x;
+        }
+        if (tid < B && (tid & 31) == 31) qs[B + 4 + (tid >> 5)] = incl;
+        if (tid == 0) qs[B + 2] = -1;
+        G::sync();
+        if (tid < B) {
+            int before = 0;
+            for (int w = 0; w < (tid >> 5); ++w) before += qs[B + 4 + w];
+            incl += before;
+            if (incl - v < need && need <= incl) {  // exactly one thread: its bin holds the wanted rank
+                qs[B + 2] = tid;
+                qs[B + 3] = incl;
+                qs[B + 36] = v;
+            }
+        }
+        G::sync();
+        bin = qs[B + 2];
+        incl_total = qs[B + 3];
+        bin_count = qs[B + 36];
+        G::sync();  // everybody has read the result and the warp sums
+        if (tid < B) qs[tid] = 0;
+        if (tid < kQuickWords - B) qs[B + tid] = (tid == 0) ? -1 : 0;
+        G::sync();
+    };
+    // bins of the distance bits: (distance - base) >> sh, when that is below B
+    auto dist_bin = [&](unsigned base, int sh) {
+        return [=](unsigned long long key) {
+            const unsigned h = (unsigned)(key >> 32);
+            if (h < base) return -1;
+            const unsigned b = (h - base) >> sh;
+            return b < (unsigned)B ? (int)b : -1;
+        };
+    };
+
+    hist_pass(dist_bin(lo, shift), k);
+    int below = incl_total - bin_count;   // keys in the bins before the boundary bin
+    unsigned base = lo;                   // first distance of the boundary bin is base + (bin << sh)
+    int sh = shift;
+    // exclusive bound on the keys that stay
+    unsigned long long bound = ((unsigned long long)base + ((unsigned long long)(bin + 1) << sh)) << 32;
+    bool ok = bin >= 0;
+    if (REFINE) {
+        // narrow the distance bits while the boundary bin is crowded
+        for (int level = 0; level < 3 && ok && below + bin_count > keep_max && sh > 0; ++level) {
+            base += (unsigned)bin << sh;
+            sh = sh > 8 ? sh - 8 : 0;
+            hist_pass(dist_bin(base, sh), k - below);
+            ok = bin >= 0;
+            below += incl_total - bin_count;
+            bound = ((unsigned long long)base + ((unsigned long long)(bin + 1) << sh)) << 32;
+        }
+        if (ok && below + bin_count > keep_max && bin_count > 1 && sh == 0) {
+            // many keys share one distance (base + bin): split that group by the low word (the id)
+            const unsigned tie = base + (unsigned)bin;
+            unsigned ilo = 0xFFFFFFFFu, ihi = 0u;
+#pragma unroll
+            for (int j = 0; j < kPerThread; ++j) {
+                const int i = tid + j * NT;
+                if (i < n && (unsigned)(mine[j] >> 32) == tie) {
+                    ilo = min(ilo, (unsigned)mine[j]);
+                    ihi = max(ihi, (unsigned)mine[j]);
+                }
+            }
+            ilo = __reduce_min_sync(0xFFFFFFFFu, ilo);
+            ihi = __reduce_max_sync(0xFFFFFFFFu, ihi);
+            if ((tid & 31) == 0) {
+                atomicMin(&uq[B], ilo);
+                atomicMax(&uq[B + 1], ihi);
+            }
+            G::sync();
+            ilo = uq[B];
+            ihi = uq[B + 1];
+            G::sync();
+            if (tid == 0) {
+                uq[B] = 0xFFFFFFFFu;
+                uq[B + 1] = 0u;
+            }
+            const unsigned irange = ihi - ilo;
+            int ish = 0;
+            if (irange >= (unsigned)B) ish = (32 - __clz(irange)) - (31 - __clz(B));
+            G::sync();
+            hist_pass([=](unsigned long long key) {
+                return (unsigned)(key >> 32) == tie ? (int)(((unsigned)key - ilo) >> ish) : -1;
+            }, k - below);
+            ok = bin >= 0;
+            below += incl_total - bin_count;
+            const unsigned long long next_id = (unsigned long long)ilo + ((unsigned long long)(bin + 1) << ish);
+            bound = next_id > 0xFFFFFFFFull ? ((unsigned long long)tie + 1ull) << 32 : ((unsigned long long)tie << 32) | next_id;
         }
     }
-    G::sync();
-    const int bstar = qs[B + 2];
-    const int kept = qs[B + 3];
-    G::sync();  // everybody has read the result and the warp sums
-    if (tid < B) qs[tid] = 0;  // back to the all-zero state for the next call
-    if (tid < kQuickWords - B) qs[B + tid] = (tid == 0) ? -1 : 0;
-    if (kept >= n) {  // uniform: nothing would be dropped
-        G::sync();
+    const int kept = below + bin_count;
+    if (!ok || kept >= n) {  // uniform: nothing would be dropped
         topk_select<NT, G, CAP>(t, k);  // uses the same shared words as its histogram
         topk_quick_init<NT, G>(qs);
         return;
     }
-    // exclusive bound on the keys that stay
-    const unsigned long long bound = ((unsigned long long)lo + ((unsigned long long)(bstar + 1) << shift)) << 32;
     if (tid == 0) {
         *t.cnt = 0;
         *t.tau = bound < kKeyPad ? bound : kKeyPad;
