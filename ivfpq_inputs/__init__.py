@@ -4,7 +4,8 @@ This package is test/bench infrastructure shared by the CPU oracle's tests and
 by the CUDA library's tests: it draws the synthetic base vectors and queries,
 trains and encodes an IVFPQ index from them (the paper's offline phase,
 Algorithm 1, without the ray-tracing scene and without the entry->points map),
-calibrates hit radii, computes exact brute-force neighbours for recall, and
+calibrates hit radii, builds the density maps and the polynomial regressor of the dynamic
+threshold, computes exact brute-force neighbours for recall, and
 reads/writes the index file.  It contains none of the online search steps
 (coarse probe selection, selective look-up table, list scan, top-k): those live
 in `oracle/` (CPU) and in the CUDA library, which share no code.
@@ -22,6 +23,7 @@ from .index_build import (
     save_index,
 )
 from .groundtruth import exact_knn, recall_at_k, recall_1_at_k
+from .thresholds import ThresholdModel, containing_thresholds, density_maps, fit_threshold_model
 
 __all__ = [
     "CONFIGS",
@@ -40,4 +42,8 @@ __all__ = [
     "exact_knn",
     "recall_at_k",
     "recall_1_at_k",
+    "ThresholdModel",
+    "containing_thresholds",
+    "density_maps",
+    "fit_threshold_model",
 ]

@@ -63,6 +63,8 @@ def _lib() -> ctypes.CDLL:
                                       vp, vp,                                          # outputs
                                       vp, vp, vp, vp, i64, vp, vp, vp]                 # dumps
         lib.oracle_search.restype = i32
+        lib.oracle_thresholds.argtypes = [i32, i32, i32, vp, i64, i32, i32, vp, vp, vp, vp, vp]
+        lib.oracle_thresholds.restype = i32
         lib.oracle_num_threads.restype = i32
         lib.oracle_set_num_threads.argtypes = [i32]
         _LIB = lib
@@ -150,3 +152,20 @@ def search(index, queries: np.ndarray, nprobe: int, k: int, *, dense: bool = Fal
     if rc != 0:
         raise ValueError(f"oracle_search failed: {rc}")
     return res
+
+
+def thresholds(d: int, nsub: int, dsub: int, queries: np.ndarray, model) -> np.ndarray:
+    """Dynamic thresholds [nq, nsub] fp32 from a density-map + polynomial model (an object with
+    `grid`, `degree`, `density` [nsub, grid, grid], `origin` [nsub, 2], `inv_cell` [nsub, 2] and
+    `coef` [nsub, degree + 1], as `ivfpq_inputs.ThresholdModel`)."""
+    q = _c(queries, np.float32)
+    dens = _c(model.density, np.float32)
+    org = _c(model.origin, np.float32)
+    inv = _c(model.inv_cell, np.float32)
+    cf = _c(model.coef, np.float32)
+    out = np.empty((q.shape[0], nsub), np.float32)
+    rc = _lib().oracle_thresholds(d, nsub, dsub, _p(q), q.shape[0], int(model.grid), int(model.degree),
+                                  _p(dens), _p(org), _p(inv), _p(cf), _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle_thresholds failed: {rc}")
+    return out

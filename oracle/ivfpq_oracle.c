@@ -28,6 +28,11 @@
  *   S4  the k smallest (distance, id) pairs, ascending (Sec. 2.1, last paragraph).
  * Dense search is the same with every entry selected.
  *
+ * Before S2, the query-specific thresholds can come from the dynamic threshold front-end (Sec. 3.1
+ * "Determining Proper Threshold"; Algorithm 2, line 5): oracle_thresholds() below looks up the
+ * density of the grid cell the query's projection falls into and evaluates the polynomial
+ * regressor on it.
+ *
  * Parity pins (tests/test_oracle_pins.py): radius -> inf equals dense bit for bit;
  * dense distance equals the fp64 distance to the reconstructed vector; a lossless
  * toy index reproduces brute-force exact neighbours; nesting/monotonicity in radius
@@ -240,4 +245,44 @@ int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* c
         free(scratch);
     }
     return status;
+}
+
+/*
+ * Dynamic thresholds (Sec. 3.1 "Determining Proper Threshold": every 2-d subspace is divided into a
+ * grid x grid map of cell densities; "during runtime, we look up the density of the query
+ * projection in each subspace and use the regression model to infer a query-specific threshold";
+ * Algorithm 2, line 5: thres = poly_regressor(density_map(x, y)) with (x, y) the query's own
+ * projection, taken before the centroid is subtracted).
+ *   density  [nsub][grid][grid]   row = cell index along the second coordinate, column = first
+ *   origin   [nsub][2]            lower corner of the grid
+ *   inv_cell [nsub][2]            1 / cell size along each coordinate
+ *   coef     [nsub][degree+1]     polynomial coefficients, ascending powers of the density
+ *   radius   [nq][nsub]           out: max(0, polynomial(density of the cell)); projections outside the
+ *                                 grid use the nearest border cell
+ * fp32: cell = floor((x - origin) * inv_cell); Horner evaluation with fmaf from the highest power.
+ */
+int oracle_thresholds(int d, int nsub, int dsub, const float* queries, int64_t nq, int grid, int degree,
+                      const float* density, const float* origin, const float* inv_cell, const float* coef,
+                      float* radius) {
+    if (dsub != 2 || d != nsub * dsub || grid <= 0 || degree < 0) return -2;
+    for (int64_t qi = 0; qi < nq; ++qi) {
+        for (int s = 0; s < nsub; ++s) {
+            int cell[2];
+            for (int a = 0; a < 2; ++a) {
+                float t = (queries[qi * d + 2 * s + a] - origin[2 * s + a]) * inv_cell[2 * s + a];
+                float f = floorf(t);
+                int c = 0;
+                if (f >= (float)grid) c = grid - 1;
+                else if (f > 0.0f) c = (int)f;      /* NaN and negatives stay at 0 */
+                if (c > grid - 1) c = grid - 1;
+                cell[a] = c;
+            }
+            const float dens = density[((size_t)s * grid + cell[1]) * grid + cell[0]];
+            const float* cf = coef + (size_t)s * (degree + 1);
+            float acc = cf[degree];
+            for (int i = degree - 1; i >= 0; --i) acc = fmaf(acc, dens, cf[i]);
+            radius[qi * nsub + s] = acc > 0.0f ? acc : 0.0f;
+        }
+    }
+    return 0;
 }
