@@ -97,6 +97,32 @@ typedef struct {
     float miss_penalty;
 } ivfpq_radius_t;
 
+/* Dynamic threshold model (Sec. 3.1 "Determining Proper Threshold"): per 2-d subspace a grid x grid
+ * map of cell densities (number of base projections in the cell / cell area) and a polynomial that
+ * maps a density to a threshold.  All arrays are device memory owned by the caller. */
+typedef struct {
+    int32_t grid;          /* cells per axis, 1..4096 (the paper uses 100)                        */
+    int32_t degree;        /* polynomial degree, 0..8                                              */
+    const float* density;  /* dev [nsub][grid][grid]: row = cell along the second coordinate       */
+    const float* origin;   /* dev [nsub][2]: lower corner of the grid, 8-byte aligned              */
+    const float* inv_cell; /* dev [nsub][2]: 1 / cell size along each coordinate, 8-byte aligned   */
+    const float* coef;     /* dev [nsub][degree + 1]: coefficients, ascending powers               */
+} ivfpq_threshold_model_t;
+
+/* Query-specific thresholds (Algorithm 2, line 5: thres = poly_regressor(density_map(x, y))):
+ * radius_out[q][s] = max(0, polynomial_s(density_s[cell of (queries[q][2s], queries[q][2s+1])])),
+ * cell = floor((coordinate - origin) * inv_cell) clamped to the grid (an undefined coordinate falls
+ * into cell 0).  The projection is the query's own (the centroid is not subtracted, as in
+ * Algorithm 2).  The polynomial is evaluated in fp32 by Horner's rule from the highest power, one
+ * fused multiply-add per coefficient.  The result is the radius array of ivfpq_search_sparse in
+ * mode 1 ([nq][nsub], before the user's scale).  Only for indexes with 2-d subspaces (dsub == 2,
+ * the paper's setting), grid and degree within the limits above and nq <= 2^24:
+ * IVFPQ_ERR_UNSUPPORTED otherwise; null or misaligned pointers: IVFPQ_ERR_INVALID_ARGUMENT.
+ * queries dev [nq][d], 8-byte aligned; radius_out dev [nq][nsub].  Asynchronous on `stream`;
+ * allocates nothing. */
+int ivfpq_query_thresholds(const ivfpq_index_t* index, const float* queries, int64_t nq,
+                           const ivfpq_threshold_model_t* model, float* radius_out, void* stream);
+
 /* Workspace (dev, 256-byte aligned) needed by one search call of this shape. */
 size_t ivfpq_search_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k);
 

@@ -35,7 +35,7 @@ EXPORTS = (
     "ivfpq_search_workspace_bytes", "ivfpq_search_dense", "ivfpq_search_sparse",
     "ivfpq_search_host_workspace_bytes", "ivfpq_search_host", "ivfpq_sync_status",
     "ivfpq_index_set_option", "ivfpq_last_launch_count", "ivfpq_last_stage_ms", "ivfpq_error_string",
-    "ivfpq_debug_probes", "ivfpq_debug_search", "ivfpq_probe_static",
+    "ivfpq_debug_probes", "ivfpq_debug_search", "ivfpq_probe_static", "ivfpq_query_thresholds",
 )
 
 
@@ -56,6 +56,11 @@ class ivfpq_index_desc_t(ctypes.Structure):
 class ivfpq_radius_t(ctypes.Structure):
     _fields_ = [("radius", ctypes.c_void_p), ("mode", ctypes.c_int32), ("scale", ctypes.c_float),
                 ("miss_penalty", ctypes.c_float)]
+
+
+class ivfpq_threshold_model_t(ctypes.Structure):
+    _fields_ = [("grid", ctypes.c_int32), ("degree", ctypes.c_int32), ("density", ctypes.c_void_p),
+                ("origin", ctypes.c_void_p), ("inv_cell", ctypes.c_void_p), ("coef", ctypes.c_void_p)]
 
 
 _lib: Optional[ctypes.CDLL] = None
@@ -102,6 +107,8 @@ def load_library() -> ctypes.CDLL:
     lib.ivfpq_debug_search.argtypes = [vp, vp, i64, i32, ctypes.POINTER(ivfpq_radius_t), i32, vp, vp,
                                        vp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
     lib.ivfpq_debug_search.restype = ctypes.c_int
+    lib.ivfpq_query_thresholds.argtypes = [vp, vp, i64, ctypes.POINTER(ivfpq_threshold_model_t), vp, vp]
+    lib.ivfpq_query_thresholds.restype = ctypes.c_int
     lib.ivfpq_probe_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
     lib.ivfpq_probe_static.restype = ctypes.c_int
     _lib = lib
@@ -340,3 +347,29 @@ def ivfpq_probe_static(ix: IndexHandle, queries: torch.Tensor, nprobe: int,
     _check(load_library().ivfpq_probe_static(ix.handle, queries.data_ptr(), nq, nprobe, pid.data_ptr(),
                                              pd.data_ptr(), _stream()), "ivfpq_probe_static")
     return pid, pd
+
+
+class ThresholdModelHandle:
+    """Device copies of a dynamic threshold model (an object with grid, degree, density
+    [nsub, grid, grid], origin [nsub, 2], inv_cell [nsub, 2], coef [nsub, degree + 1])."""
+
+    def __init__(self, model, device="cuda"):
+        f = lambda a: torch.from_numpy(np.ascontiguousarray(a, np.float32)).to(device)
+        self.grid, self.degree = int(model.grid), int(model.degree)
+        self.density, self.origin, self.inv_cell, self.coef = f(model.density), f(model.origin), f(model.inv_cell), f(model.coef)
+        self.struct = ivfpq_threshold_model_t(self.grid, self.degree, self.density.data_ptr(), self.origin.data_ptr(),
+                                              self.inv_cell.data_ptr(), self.coef.data_ptr())
+
+
+def ivfpq_query_thresholds(ix: IndexHandle, queries: torch.Tensor, model: ThresholdModelHandle,
+                           out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Query-specific thresholds [nq, nsub] fp32 on the device (the mode-1 radius of the sparse search)."""
+    if queries.dtype != torch.float32 or not queries.is_cuda or not queries.is_contiguous() or queries.dim() != 2 \
+            or queries.shape[1] != ix.d:
+        raise ValueError("queries must be a contiguous fp32 CUDA tensor [nq, d]")
+    nq = queries.shape[0]
+    if out is None:
+        out = torch.empty((nq, ix.nsub), dtype=torch.float32, device=queries.device)
+    _check(load_library().ivfpq_query_thresholds(ix.handle, queries.data_ptr(), nq, ctypes.byref(model.struct),
+                                                 out.data_ptr(), _stream()), "ivfpq_query_thresholds")
+    return out

@@ -264,6 +264,19 @@ int ivfpq_index_free(ivfpq_index_t* index) {
     return IVFPQ_OK;
 }
 
+int ivfpq_query_thresholds(const ivfpq_index_t* index, const float* queries, int64_t nq,
+                           const ivfpq_threshold_model_t* model, float* radius_out, void* stream) {
+    if (!index || !queries || !model || !radius_out || nq <= 0) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (!model->density || !model->origin || !model->inv_cell || !model->coef) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (index->dsub != 2) return IVFPQ_ERR_UNSUPPORTED;
+    if (model->grid < 1 || model->grid > 4096 || model->degree < 0 || model->degree > 8) return IVFPQ_ERR_UNSUPPORTED;
+    if (nq > (int64_t)1 << 24) return IVFPQ_ERR_UNSUPPORTED;
+    if (!aligned(queries, 8) || !aligned(model->origin, 8) || !aligned(model->inv_cell, 8)) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (launch_thresholds(queries, nq, index->nsub, model, radius_out, reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    return IVFPQ_OK;
+}
+
 size_t ivfpq_search_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k) {
     if (check_search_shape(index, nq, nprobe, k) != IVFPQ_OK) return 0;
     return plan_workspace(index, nq, nprobe, k).total;
