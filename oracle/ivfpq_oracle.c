@@ -28,6 +28,17 @@
  *   S4  the k smallest (distance, id) pairs, ascending (Sec. 2.1, last paragraph).
  * Dense search is the same with every entry selected.
  *
+ * Hit-count scores (Sec. 4.4 "Aggressive Approximation: hit count-based Method"; the -L and -M
+ * configurations of the evaluation plan in Sec. 5.1) replace S3's distance by a count, S1, S2's
+ * selection and S4 unchanged:
+ *   score 1 (hit count): a point is ranked by the number of subspaces in which its entry was
+ *       selected, more hits first.  Reported value: the number of subspaces missed (nsub - hits),
+ *       so that smaller is better as for distances.
+ *   score 2 (reward / penalty): every sphere gets an inner sphere of half the radius; a subspace
+ *       adds +1 when the entry lies within the inner sphere, -1 when it lies outside the outer
+ *       one, 0 in between; more is better.  Reported value: nsub - score (0, 1 or 2 per subspace).
+ *   The inner test is d2 <= 0.25f * (radius*scale)^2 on the same squared distance.
+ *
  * Before S2, the query-specific thresholds can come from the dynamic threshold front-end (Sec. 3.1
  * "Determining Proper Threshold"; Algorithm 2, line 5): oracle_thresholds() below looks up the
  * density of the grid cell the query's projection falls into and evaluates the polynomial
@@ -124,17 +135,20 @@ int oracle_coarse(const float* queries, int64_t nq, int d, const float* cent, in
  *   row = entry e selected); visit_count [nq]; and, with visit_stride slots per query in
  *   visiting order (probe rank, then position in the list): visit_hits (bit s = subspace
  *   s selected for that point), visit_dist, visit_ids.
+ * score: 0 = distances (S3 as above), 1 = hit count, 2 = reward / penalty (header comment); the
+ *   two count scores need a radius (not dense).
  */
-int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* cent,
+int oracle_search_scored(int d, int nlist, int nsub, int dsub, int ksub, const float* cent,
                   const float* codebooks, const int64_t* list_offsets, const uint8_t* codes,
                   const int32_t* ids, const float* queries, int64_t nq, int nprobe, int dense,
-                  const float* radius, int radius_mode, float scale, float miss_penalty, int k,
+                  const float* radius, int radius_mode, float scale, float miss_penalty, int score, int k,
                   float* out_dist, int32_t* out_ids, int32_t* probe_ids_out, float* probe_d_out,
                   uint32_t* masks_out, int64_t* visit_count, int64_t visit_stride,
                   uint64_t* visit_hits, float* visit_dist, int32_t* visit_ids) {
     if (d != nsub * dsub || ksub <= 0 || ksub > 256 || nsub > 64) return -2;
     if (nprobe <= 0 || nprobe > nlist || k <= 0) return -1;
     if (!dense && radius == NULL) return -1;
+    if (score < 0 || score > 2 || (dense && score != 0)) return -1;
     int status = 0;
 
 #pragma omp parallel
@@ -184,6 +198,8 @@ int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* c
                             d2 = fmaf(t, t, d2);
                         }
                         int h = dense ? 1 : (d2 <= r2[s]);
+                        /* level 2: also within the inner sphere of half the radius */
+                        if (h && score == 2 && d2 <= 0.25f * r2[s]) h = 2;
                         lut[(size_t)s * ksub + e] = d2;
                         hit[(size_t)s * ksub + e] = (uint8_t)h;
                         if (h) mrow[e >> 5] |= 1u << (e & 31);
@@ -196,17 +212,22 @@ int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* c
                     const uint8_t* code = codes + (size_t)x * nsub;
                     float S = 0.0f;
                     int m = 0;
+                    int reward = 0; /* score 2: +1 inner hit, -1 missed both spheres */
                     uint64_t hs = 0;
                     for (int s = 0; s < nsub; ++s) {
                         int e = code[s];
                         if (e < ksub && hit[(size_t)s * ksub + e]) {
                             S = S + lut[(size_t)s * ksub + e];
                             hs |= (uint64_t)1 << s;
+                            if (hit[(size_t)s * ksub + e] == 2) reward += 1;
                         } else {
                             m += 1;
+                            reward -= 1;
                         }
                     }
                     float dist = (m == 0) ? S : fmaf((float)m, P, S);
+                    if (score == 1) dist = (float)m;
+                    if (score == 2) dist = (float)(nsub - reward);
                     if (n == cap) {
                         cap *= 2;
                         vis = (cand_t*)realloc(vis, sizeof(cand_t) * cap);
@@ -247,10 +268,23 @@ int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* c
     return status;
 }
 
+int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* cent,
+                  const float* codebooks, const int64_t* list_offsets, const uint8_t* codes,
+                  const int32_t* ids, const float* queries, int64_t nq, int nprobe, int dense,
+                  const float* radius, int radius_mode, float scale, float miss_penalty, int k,
+                  float* out_dist, int32_t* out_ids, int32_t* probe_ids_out, float* probe_d_out,
+                  uint32_t* masks_out, int64_t* visit_count, int64_t visit_stride,
+                  uint64_t* visit_hits, float* visit_dist, int32_t* visit_ids) {
+    return oracle_search_scored(d, nlist, nsub, dsub, ksub, cent, codebooks, list_offsets, codes, ids, queries, nq,
+                                nprobe, dense, radius, radius_mode, scale, miss_penalty, 0, k, out_dist, out_ids,
+                                probe_ids_out, probe_d_out, masks_out, visit_count, visit_stride, visit_hits,
+                                visit_dist, visit_ids);
+}
+
 /*
  * Dynamic thresholds (Sec. 3.1 "Determining Proper Threshold": every 2-d subspace is divided into a
- * grid x grid map of cell densities; "during runtime, we look up the density of the query
- * projection in each subspace and use the regression model to infer a query-specific threshold";
+ * grid x grid map of cell densities; at search time the density of the cell that holds the query's
+ * projection is read and a regression polynomial turns it into that query's threshold;
  * Algorithm 2, line 5: thres = poly_regressor(density_map(x, y)) with (x, y) the query's own
  * projection, taken before the centroid is subtracted).
  *   density  [nsub][grid][grid]   row = cell index along the second coordinate, column = first
