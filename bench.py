@@ -165,6 +165,22 @@ def pick_scale(search_sparse, search_dense, true_ids, scales=(0.5, 0.75, 1.0, 1.
     return r_dense, recall_1_at_k(dense_ids, true_ids), chosen, table
 
 
+def pick_scale_for_counts(search_sparse, true_ids, scales=(0.5, 0.75, 1.0, 1.25, 1.5, 2.0, 3.0)):
+    """Count scores never reproduce the dense ranking: take the radius scale with the best R1@100
+    (the paper's quality measure for its hit-count configurations, Sec. 5.1)."""
+    best, table = None, []
+    for s in scales:
+        ids = search_sparse(s)
+        r, r1 = recall_at_k(ids, true_ids), recall_1_at_k(ids, true_ids)
+        table.append((s, round(r, 4), round(r1, 4)))
+        if best is None or r1 > best[2]:
+            best = (s, r, r1)
+    return best, table
+
+
+SCORE_NAMES = {"distance": 0, "hit_count": 1, "reward_penalty": 2}
+
+
 def scan_kernel_name(index) -> str:
     """Name of the kernel the library picks for this index (same rule as ivfpq_index_load)."""
     if (index.nsub, index.dsub) == (16, 8):
@@ -215,10 +231,14 @@ def run_cuda(args):
     def dense_ids():
         return lib.ivfpq_search_dense(h, qd, nprobe, k)[1].cpu().numpy()
 
+    score = SCORE_NAMES[args.score]
+
     def sparse_ids(s):
-        return lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=s)[1].cpu().numpy()
+        return lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=s, score=score)[1].cpu().numpy()
 
     r_dense, r1_dense, (scale, r_sparse, r1_sparse), sweep = pick_scale(sparse_ids, dense_ids, true_ids)
+    if score != 0:
+        (scale, r_sparse, r1_sparse), sweep = pick_scale_for_counts(sparse_ids, true_ids)
     assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
     log(f"[bench] recall@100 dense {r_dense:.4f}, sparse {r_sparse:.4f} at scale {scale} (sweep {sweep})")
 
@@ -230,7 +250,7 @@ def run_cuda(args):
     lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_TIMING, 1)
 
     def step_sparse():
-        lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=scale, out=out)
+        lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=scale, out=out, score=score)
 
     def step_dense():
         lib.ivfpq_search_dense(h, qd, nprobe, k, out=out)
@@ -272,7 +292,7 @@ def run_cuda(args):
     oih = torch.empty((nq, k), dtype=torch.int32).pin_memory()
 
     def step_host():
-        lib.ivfpq_search_host(h, qh, nprobe, k, odh, oih, radius=rad_d, scale=scale)
+        lib.ivfpq_search_host(h, qh, nprobe, k, odh, oih, radius=rad_d, scale=scale, score=score)
 
     lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_TIMING, 0)
     e2e_steps = max(3, args.steps // 4)
@@ -298,7 +318,7 @@ def run_cuda(args):
     gather_peak = props.multi_processor_count * 32 * clk * 1e6 / 1e9            # G gathers/s
     gather_rate = scan_bytes / (scan_ms * 1e-3) / 1e9                            # one gather per code byte
 
-    cpu = cpu_baseline(index, q_np, nprobe, k, radius, scale, args.cpu_sample)
+    cpu = cpu_baseline(index, q_np, nprobe, k, radius, scale, args.cpu_sample, score)
 
     line = {
         "metric": METRIC, "value": nq * world * args.steps / (total_ms * 1e-3), "unit": UNIT,
@@ -306,10 +326,11 @@ def run_cuda(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{cfg.name}: N={index.ntotal} D={index.d} nlist={index.nlist} "
                                f"PQ {index.nsub}x{index.dsub} (uint8 codes), nq={nq}/GPU, nprobe={nprobe}, k={k}, "
-                               f"sparse search at radius scale {scale}",
+                               f"sparse search at radius scale {scale}"
+                               + ("" if score == 0 else f", ranked by {args.score}"),
                    "l2": "512 MiB buffer written between timed iterations (L2 flush)",
                    "parallelism": "replicas only (index replicated, queries split)" if world > 1 else "1 GPU",
-                   "radius_scale": scale, "nprobe": nprobe},
+                   "radius_scale": scale, "nprobe": nprobe, "score": args.score},
         "recall@100": {"sparse": round(r_sparse, 4), "dense": round(r_dense, 4),
                        "R1@100_sparse": round(r1_sparse, 4), "R1@100_dense": round(r1_dense, 4)},
         "dense_queries_per_s": nq * world * dense_steps / (dense_ms * 1e-3),
@@ -323,7 +344,8 @@ def run_cuda(args):
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_source": f"of {peak_src}", "algorithmic_bytes_per_launch": int(scan_bytes),
                      "visits_per_launch": int(visits),
-                     "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload) if (args.nq is None and args.nprobe == 0) else None},
+                     "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload)
+                     if (args.nq is None and args.nprobe == 0 and score == 0) else None},
         "gather_roofline": {"bound": "shared-memory gathers", "achieved": gather_rate, "peak": gather_peak,
                             "unit": "Ggather/s", "frac": gather_rate / gather_peak,
                             "peak_source": f"{props.multi_processor_count} SMs x 32 lanes x {clk:.0f} MHz"},
@@ -346,12 +368,12 @@ class _Null:
 # the CPU oracle: cpu_baseline leg and --impl reference
 # --------------------------------------------------------------------------------------------
 
-def cpu_baseline(index, q_np, nprobe, k, radius, scale, sample):
+def cpu_baseline(index, q_np, nprobe, k, radius, scale, sample, score=0):
     import oracle
     sample = min(sample, q_np.shape[0])
-    oracle.search(index, q_np[:8], nprobe, k, radius=radius, scale=scale)    # page in
+    oracle.search(index, q_np[:8], nprobe, k, radius=radius, scale=scale, score=score)    # page in
     t0 = time.perf_counter()
-    oracle.search(index, q_np[:sample], nprobe, k, radius=radius, scale=scale)
+    oracle.search(index, q_np[:sample], nprobe, k, radius=radius, scale=scale, score=score)
     dt = time.perf_counter() - t0
     return {"value": sample / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
             "sample": f"first {sample} queries of the batch, one oracle.search call, {dt:.2f} s"}
@@ -403,6 +425,8 @@ def main():
     ap.add_argument("--nq", type=int, default=None)
     ap.add_argument("--cpu-sample", type=int, default=10000, help="queries timed on the CPU oracle")
     ap.add_argument("--ref-scale", type=float, default=1.0)
+    ap.add_argument("--score", default="distance", choices=sorted(SCORE_NAMES),
+                    help="what the sparse search ranks by (distance = the headline path)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3

@@ -89,12 +89,29 @@ int ivfpq_index_free(ivfpq_index_t* index);
  * thres_scale in Algorithm 2); an entry is selected when its squared distance to the residual
  * projection is <= (radius*scale)^2.  miss_penalty is the constant P added per subspace whose
  * entry was not selected; a negative value asks for the default P = sum over subspaces of
- * (radius*scale)^2 of that query, which ranks points first by number of missed subspaces. */
+ * (radius*scale)^2 of that query, which ranks points first by number of missed subspaces.
+ *
+ * `score` chooses what a point is ranked by (Sec. 4.4 "Aggressive Approximation: hit count-based
+ * Method"; the -H / -L / -M configurations of Sec. 5.1).  Selection, probing and the top-k rule
+ * ((value, id) ascending, padded with (+inf, -1)) are the same for all three:
+ *   IVFPQ_SCORE_DISTANCE        value = S + m * P as described above (miss_penalty applies).
+ *   IVFPQ_SCORE_HIT_COUNT       value = number of subspaces whose entry was NOT selected
+ *                               (nsub - hit count): more hits rank first.
+ *   IVFPQ_SCORE_REWARD_PENALTY  every sphere has an inner sphere of half the radius; per subspace
+ *                               0 when the entry is within the inner sphere (reward +1), 1 when only
+ *                               within the outer one, 2 when outside both (penalty -1);
+ *                               value = the sum = nsub - (rewards - penalties).  Inner test:
+ *                               squared distance <= 0.25f * (radius*scale)^2.
+ * The count values are small integers, exact in fp32; miss_penalty is ignored for them. */
+#define IVFPQ_SCORE_DISTANCE 0
+#define IVFPQ_SCORE_HIT_COUNT 1
+#define IVFPQ_SCORE_REWARD_PENALTY 2
 typedef struct {
     const float* radius; /* dev; mode 0: [nsub], mode 1: [nq][nsub] */
     int32_t mode;
     float scale;
     float miss_penalty;
+    int32_t score;       /* IVFPQ_SCORE_*; other values: IVFPQ_ERR_INVALID_ARGUMENT */
 } ivfpq_radius_t;
 
 /* Dynamic threshold model (Sec. 3.1 "Determining Proper Threshold"): per 2-d subspace a grid x grid

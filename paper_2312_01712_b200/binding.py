@@ -29,6 +29,9 @@ IVFPQ_STATIC_SCRATCH_BYTES = 8 << 20
 IVFPQ_STATIC_MAX_NLIST = 16384
 IVFPQ_OPT_NSPLIT = 1
 IVFPQ_OPT_TIMING = 2
+IVFPQ_SCORE_DISTANCE = 0
+IVFPQ_SCORE_HIT_COUNT = 1
+IVFPQ_SCORE_REWARD_PENALTY = 2
 
 EXPORTS = (
     "ivfpq_index_derived_bytes", "ivfpq_index_load", "ivfpq_index_free",
@@ -55,7 +58,7 @@ class ivfpq_index_desc_t(ctypes.Structure):
 
 class ivfpq_radius_t(ctypes.Structure):
     _fields_ = [("radius", ctypes.c_void_p), ("mode", ctypes.c_int32), ("scale", ctypes.c_float),
-                ("miss_penalty", ctypes.c_float)]
+                ("miss_penalty", ctypes.c_float), ("score", ctypes.c_int32)]
 
 
 class ivfpq_threshold_model_t(ctypes.Structure):
@@ -209,7 +212,8 @@ def ivfpq_search_workspace_bytes(ix: IndexHandle, nq: int, nprobe: int, k: int) 
     return int(load_library().ivfpq_search_workspace_bytes(ix.handle, nq, nprobe, k))
 
 
-def _radius_struct(ix: IndexHandle, nq: int, radius: torch.Tensor, scale: float, miss_penalty: float):
+def _radius_struct(ix: IndexHandle, nq: int, radius: torch.Tensor, scale: float, miss_penalty: float,
+                   score: int = IVFPQ_SCORE_DISTANCE):
     if radius.dtype != torch.float32 or not radius.is_cuda or not radius.is_contiguous():
         raise ValueError("radius must be a contiguous fp32 CUDA tensor")
     if tuple(radius.shape) == (ix.nsub,):
@@ -218,7 +222,7 @@ def _radius_struct(ix: IndexHandle, nq: int, radius: torch.Tensor, scale: float,
         mode = 1
     else:
         raise ValueError("radius must be [nsub] or [nq, nsub]")
-    return ivfpq_radius_t(radius.data_ptr(), mode, float(scale), float(miss_penalty))
+    return ivfpq_radius_t(radius.data_ptr(), mode, float(scale), float(miss_penalty), int(score))
 
 
 def _prep(ix: IndexHandle, queries: torch.Tensor, nprobe: int, k: int):
@@ -251,12 +255,14 @@ def ivfpq_search_dense(ix: IndexHandle, queries: torch.Tensor, nprobe: int, k: i
 
 def ivfpq_search_sparse(ix: IndexHandle, queries: torch.Tensor, nprobe: int, radius: torch.Tensor, k: int,
                         scale: float = 1.0, miss_penalty: float = -1.0,
-                        out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None):
-    """Sparsity-aware search with per-subspace threshold radii."""
+                        out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None,
+                        score: int = IVFPQ_SCORE_DISTANCE):
+    """Sparsity-aware search with per-subspace threshold radii; `score` = IVFPQ_SCORE_DISTANCE,
+    IVFPQ_SCORE_HIT_COUNT or IVFPQ_SCORE_REWARD_PENALTY."""
     nq, ws, out_d, out_i = _prep(ix, queries, nprobe, k)
     if out is not None:
         out_d, out_i = out
-    rs = _radius_struct(ix, nq, radius, scale, miss_penalty)
+    rs = _radius_struct(ix, nq, radius, scale, miss_penalty, score)
     _check(load_library().ivfpq_search_sparse(ix.handle, queries.data_ptr(), nq, nprobe, ctypes.byref(rs), k,
                                               out_d.data_ptr(), out_i.data_ptr(), ws.data_ptr(), ws.numel(),
                                               _stream()), "ivfpq_search_sparse")
@@ -265,7 +271,8 @@ def ivfpq_search_sparse(ix: IndexHandle, queries: torch.Tensor, nprobe: int, rad
 
 def ivfpq_search_host(ix: IndexHandle, queries_host: torch.Tensor, nprobe: int, k: int,
                       out_dist_host: torch.Tensor, out_ids_host: torch.Tensor,
-                      radius: Optional[torch.Tensor] = None, scale: float = 1.0, miss_penalty: float = -1.0):
+                      radius: Optional[torch.Tensor] = None, scale: float = 1.0, miss_penalty: float = -1.0,
+                      score: int = IVFPQ_SCORE_DISTANCE):
     """End-to-end call with host (ideally pinned) query and result buffers; asynchronous on
     the current stream: synchronise before reading the results."""
     lib = load_library()
@@ -275,7 +282,7 @@ def ivfpq_search_host(ix: IndexHandle, queries_host: torch.Tensor, nprobe: int, 
             raise ValueError("host buffers must be contiguous CPU tensors of the right dtype")
     nbytes = int(lib.ivfpq_search_host_workspace_bytes(ix.handle, nq, nprobe, k))
     ws = ix.workspace(nbytes)
-    rs = None if radius is None else _radius_struct(ix, nq, radius, scale, miss_penalty)
+    rs = None if radius is None else _radius_struct(ix, nq, radius, scale, miss_penalty, score)
     _check(lib.ivfpq_search_host(ix.handle, queries_host.data_ptr(), nq, nprobe,
                                  None if rs is None else ctypes.byref(rs), k, out_dist_host.data_ptr(),
                                  out_ids_host.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
@@ -301,7 +308,7 @@ def ivfpq_debug_probes(ix: IndexHandle, queries: torch.Tensor, nprobe: int):
 
 def ivfpq_debug_search(ix: IndexHandle, queries: torch.Tensor, nprobe: int, k: int,
                        radius: Optional[torch.Tensor] = None, scale: float = 1.0, miss_penalty: float = -1.0,
-                       visit_stride: int = 0) -> dict:
+                       visit_stride: int = 0, score: int = IVFPQ_SCORE_DISTANCE) -> dict:
     """Search with stage dumps (test-only): probe lists, selected-entry masks and,
     per visited point, hit sets, distances and ids."""
     nq, ws, out_d, out_i = _prep(ix, queries, nprobe, k)
@@ -315,7 +322,7 @@ def ivfpq_debug_search(ix: IndexHandle, queries: torch.Tensor, nprobe: int, k: i
         vh = torch.zeros((nq, visit_stride), dtype=torch.int64, device=dev)
         vd = torch.full((nq, visit_stride), float("inf"), dtype=torch.float32, device=dev)
         vi = torch.full((nq, visit_stride), -1, dtype=torch.int32, device=dev)
-    rs = None if radius is None else _radius_struct(ix, nq, radius, scale, miss_penalty)
+    rs = None if radius is None else _radius_struct(ix, nq, radius, scale, miss_penalty, score)
     _check(load_library().ivfpq_debug_search(ix.handle, queries.data_ptr(), nq, nprobe,
                                              None if rs is None else ctypes.byref(rs), k,
                                              out_d.data_ptr(), out_i.data_ptr(), pid.data_ptr(), pd.data_ptr(),

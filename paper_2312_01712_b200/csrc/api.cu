@@ -78,6 +78,7 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
     if (!a.dense) {
         if (!a.radius || (a.radius_mode != 0 && a.radius_mode != 1)) return IVFPQ_ERR_INVALID_ARGUMENT;
         if (isnan(a.scale) || isnan(a.miss_penalty)) return IVFPQ_ERR_INVALID_ARGUMENT;
+        if (a.score < IVFPQ_SCORE_DISTANCE || a.score > IVFPQ_SCORE_REWARD_PENALTY) return IVFPQ_ERR_INVALID_ARGUMENT;
     }
     if (!aligned(a.queries, 4) || !aligned(workspace, 256)) return IVFPQ_ERR_WORKSPACE;
     if (!probes_only && !aligned(a.queries, 16)) return IVFPQ_ERR_INVALID_ARGUMENT;  // the scan kernels load rows as float4
@@ -302,6 +303,7 @@ static void fill_radius(SearchArgs& a, const ivfpq_radius_t* radius) {
     a.radius_mode = radius->mode;
     a.scale = radius->scale;
     a.miss_penalty = radius->miss_penalty;
+    a.score = radius->score;
 }
 
 int ivfpq_search_sparse(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,

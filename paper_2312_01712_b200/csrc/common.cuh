@@ -71,6 +71,7 @@ struct SearchArgs {
     int32_t radius_mode;
     float scale;
     float miss_penalty;
+    int32_t score;            // IVFPQ_SCORE_*
     float* out_dist;
     int32_t* out_ids;
     // dumps (debug build of the kernels), all optional

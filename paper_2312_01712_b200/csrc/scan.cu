@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_kernel(const ScanParams p) 
                 }
             }
             const bool hit = tid < ksub && (p.dense || d2 <= r2[s]);
-            lut[s * 256 + tid] = hit ? d2 : P;
+            lut[s * 256 + tid] = table_value(p.score, hit, d2, r2[s], P);
             if (DBG) {
                 unsigned m = __ballot_sync(0xFFFFFFFFu, hit);
                 if (lane == 0) {
@@ -319,6 +319,7 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     sp.radius_mode = a.radius_mode;
     sp.scale = a.scale;
     sp.miss_penalty = a.miss_penalty;
+    sp.score = a.dense ? IVFPQ_SCORE_DISTANCE : a.score;
     sp.dense = a.dense ? 1 : 0;
     sp.k = a.k;
     sp.nsplit = a.debug ? 1 : wl.nsplit;

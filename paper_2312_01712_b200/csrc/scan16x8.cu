@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
             }
             const int e = u + kEP * m;
             const bool hit = e < ksub && (p.dense || d2 <= thr);
-            const float val = hit ? d2 : P;
+            const float val = table_value(p.score, hit, d2, thr, P);
             unsigned char* row = lutb + m * (kEP * kRowBytes);
             *reinterpret_cast<float*>(row + st_a) = val;
             *reinterpret_cast<float*>(row + st_b) = val;

@@ -21,6 +21,7 @@ struct ScanParams {
     int radius_mode;
     float scale;
     float miss_penalty;
+    int score;   // IVFPQ_SCORE_*; 0 for the dense search
     int dense;
     int k;
     int nsplit;
@@ -37,6 +38,16 @@ struct ScanParams {
     int32_t* visit_ids;
 };
 
+// What a table slot holds for an entry at squared distance d2 from the residual projection, given
+// whether it was selected (`hit`: d2 <= thr, always true for the dense search).  Distances: the
+// squared distance, or the miss constant P (paper Sec. 4.3).  Count scores (Sec. 4.4): 0 / 1 for
+// selected / not selected; with the inner sphere of half the radius 0 / 1 / 2 for inside the inner
+// sphere / between the two / outside both.  The list scan sums slots, whatever they hold.
+__device__ __forceinline__ float table_value(int score, bool hit, float d2, float thr, float P) {
+    if (score == IVFPQ_SCORE_DISTANCE) return hit ? d2 : P;
+    if (score == IVFPQ_SCORE_HIT_COUNT) return hit ? 0.0f : 1.0f;
+    return !hit ? 2.0f : (d2 <= __fmul_rn(0.25f, thr) ? 0.0f : 1.0f);
+}
 
 // Rotated-layout scan (scan_rot.cu); returns cudaErrorNotSupported when the index shape has no
 // specialised instance.

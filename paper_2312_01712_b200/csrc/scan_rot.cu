@@ -55,7 +55,7 @@ __host__ __device__ inline size_t rot_smem_bytes(int ngroups, int d, int nprobe,
 template <int W, int DSUB, int NT, bool DBG>
 __device__ __forceinline__ void build_group(float* __restrict__ lutg, const float* __restrict__ cbt_g,
                                             const float* __restrict__ res_g, const float* __restrict__ r2_g,
-                                            int ksub, bool dense, float P, uint32_t* hitmask_g) {
+                                            int ksub, bool dense, int score, float P, uint32_t* hitmask_g) {
     constexpr int EP = NT / W;      // entries per pass
     constexpr int NCOPY = 32 / W;
     const int t = threadIdx.x;
@@ -99,7 +99,7 @@ __device__ __forceinline__ void build_group(float* __restrict__ lutg, const floa
             }
             hit = dense || d2 <= thr;
         }
-        const float val = hit ? d2 : P;
+        const float val = table_value(score, hit, d2, thr, P);
         float* row = lutg + e * 32 + c;
 #pragma unroll
         for (int it = 0; it < NCOPY; ++it) {
@@ -218,14 +218,14 @@ __global__ void __launch_bounds__(NT) scan_rot_kernel(const ScanParams p) {
         __syncthreads();
 
         // ---- selective tables, one per group ----
-        build_group<W0, DSUB, NT, DBG>(lut, p.cbt, res, r2, ksub, p.dense, P, hitmask);
+        build_group<W0, DSUB, NT, DBG>(lut, p.cbt, res, r2, ksub, p.dense, p.score, P, hitmask);
         if constexpr (W1 > 0)
             build_group<W1, DSUB, NT, DBG>(lut + kLutGroupFloats, p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
-                                           res + GR::s0(1) * DSUB, r2 + GR::s0(1), ksub, p.dense, P,
+                                           res + GR::s0(1) * DSUB, r2 + GR::s0(1), ksub, p.dense, p.score, P,
                                            hitmask + GR::s0(1) * 8);
         if constexpr (W2 > 0)
             build_group<W2, DSUB, NT, DBG>(lut + 2 * kLutGroupFloats, p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
-                                           res + GR::s0(2) * DSUB, r2 + GR::s0(2), ksub, p.dense, P,
+                                           res + GR::s0(2) * DSUB, r2 + GR::s0(2), ksub, p.dense, p.score, P,
                                            hitmask + GR::s0(2) * 8);
         __syncthreads();
         if (DBG && p.masks)
