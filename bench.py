@@ -167,7 +167,7 @@ def pick_scale(search_sparse, search_dense, true_ids, scales=(0.5, 0.75, 1.0, 1.
 
 def pick_scale_for_counts(search_sparse, true_ids, scales=(0.5, 0.75, 1.0, 1.25, 1.5, 2.0, 3.0)):
     """Count scores never reproduce the dense ranking: take the radius scale with the best R1@100
-    (the paper's quality measure for its hit-count configurations, Sec. 5.1)."""
+    (the paper's quality measure for its hit-count configurations, Sec. 6.1)."""
     best, table = None, []
     for s in scales:
         ids = search_sparse(s)

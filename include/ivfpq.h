@@ -7,11 +7,11 @@
  *   (2) L2-LUT construction for every (query, probed cluster): residual = query - centroid,
  *       squared distance from each residual projection to each codebook entry (steps B, C);
  *       in the sparsity-aware search only the entries within the threshold radius of the
- *       projection are selected (Sec. 3.1; Algorithm 2, whose ray/sphere test decides exactly
+ *       projection are selected (Sec. 4.1; Algorithm 2, whose ray/sphere test decides exactly
  *       "distance <= thres * thres_scale");
  *   (3) distance calculation: every point of a probed cluster accumulates the table values of
  *       its codes; a subspace whose entry was not selected contributes the large constant P
- *       instead (Sec. 2.1 step D; Sec. 4.3, paragraph after Algorithm 2); then the k
+ *       instead (Sec. 2.1 step D; Sec. 5.3, paragraph after Algorithm 2); then the k
  *       smallest (distance, id) pairs per query (Sec. 2.1, last paragraph).
  *
  * Naming: nsub = number of PQ subspaces (the paper's D/M), dsub = dimensions per subspace (the
@@ -91,8 +91,8 @@ int ivfpq_index_free(ivfpq_index_t* index);
  * entry was not selected; a negative value asks for the default P = sum over subspaces of
  * (radius*scale)^2 of that query, which ranks points first by number of missed subspaces.
  *
- * `score` chooses what a point is ranked by (Sec. 4.4 "Aggressive Approximation: hit count-based
- * Method"; the -H / -L / -M configurations of Sec. 5.1).  Selection, probing and the top-k rule
+ * `score` chooses what a point is ranked by (Sec. 5.4 "Aggressive Approximation: hit count-based
+ * Method"; the -H / -L / -M configurations of Sec. 6.1).  Selection, probing and the top-k rule
  * ((value, id) ascending, padded with (+inf, -1)) are the same for all three:
  *   IVFPQ_SCORE_DISTANCE        value = S + m * P as described above (miss_penalty applies).
  *   IVFPQ_SCORE_HIT_COUNT       value = number of subspaces whose entry was NOT selected
@@ -114,7 +114,7 @@ typedef struct {
     int32_t score;       /* IVFPQ_SCORE_*; other values: IVFPQ_ERR_INVALID_ARGUMENT */
 } ivfpq_radius_t;
 
-/* Dynamic threshold model (Sec. 3.1 "Determining Proper Threshold"): per 2-d subspace a grid x grid
+/* Dynamic threshold model (Sec. 4.1 "Determining Proper Threshold"): per 2-d subspace a grid x grid
  * map of cell densities (number of base projections in the cell / cell area) and a polynomial that
  * maps a density to a threshold.  All arrays are device memory owned by the caller. */
 typedef struct {
@@ -126,7 +126,7 @@ typedef struct {
     const float* coef;     /* dev [nsub][degree + 1]: coefficients, ascending powers               */
 } ivfpq_threshold_model_t;
 
-/* Query-specific thresholds (Algorithm 2, line 5: thres = poly_regressor(density_map(x, y))):
+/* Query-specific thresholds (Algorithm 2: thres = poly_regressor(density_map(x, y))):
  * radius_out[q][s] = max(0, polynomial_s(density_s[cell of (queries[q][2s], queries[q][2s+1])])),
  * cell = floor((coordinate - origin) * inv_cell) clamped to the grid (an undefined coordinate falls
  * into cell 0).  The projection is the query's own (the centroid is not subtracted, as in
@@ -150,8 +150,8 @@ int ivfpq_search_dense(const ivfpq_index_t* index, const float* queries, int64_t
                        int32_t k, float* out_dist, int32_t* out_ids, void* workspace,
                        size_t workspace_bytes, void* stream);
 
-/* Sparsity-aware search (threshold-based selective L2-LUT, Sec. 3.1 / Algorithm 2, followed
- * by the distance calculation of Sec. 4.3).  Same outputs as the dense search. */
+/* Sparsity-aware search (threshold-based selective L2-LUT, Sec. 4.1 / Algorithm 2, followed
+ * by the distance calculation of Sec. 5.3).  Same outputs as the dense search. */
 int ivfpq_search_sparse(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
                         const ivfpq_radius_t* radius, int32_t k, float* out_dist, int32_t* out_ids,
                         void* workspace, size_t workspace_bytes, void* stream);

@@ -1,6 +1,6 @@
 """Exact brute-force neighbours on the raw vectors and the recall metrics.
 
-Recall definitions follow the paper's "Metric" paragraph (Sec. 5.1): R1@k counts
+Recall definitions follow the paper's "Metric" paragraph (Sec. 6.1): R1@k counts
 the queries whose k retrieved neighbours contain the true nearest neighbour;
 recall@k here is the mean fraction of the true k nearest neighbours that were
 retrieved (the paper's R100@1000 with both numbers equal to k).

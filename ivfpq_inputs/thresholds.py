@@ -1,4 +1,4 @@
-"""Offline side of the dynamic threshold (paper Sec. 3.1 "Determining Proper Threshold"): the
+"""Offline side of the dynamic threshold (paper Sec. 4.1 "Determining Proper Threshold"): the
 per-subspace density maps and the polynomial regressor.  Harness code: it prepares the model that
 the search-time front-end (CPU oracle / CUDA library) consumes, and contains none of that front-end.
 

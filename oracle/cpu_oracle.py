@@ -69,6 +69,8 @@ def _lib() -> ctypes.CDLL:
                                              vp, vp,
                                              vp, vp, vp, vp, i64, vp, vp, vp]
         lib.oracle_search_scored.restype = i32
+        lib.oracle_entry_stats.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i64, vp, i32, vp, vp]
+        lib.oracle_entry_stats.restype = i32
         lib.oracle_thresholds.argtypes = [i32, i32, i32, vp, i64, i32, i32, vp, vp, vp, vp, vp]
         lib.oracle_thresholds.restype = i32
         lib.oracle_num_threads.restype = i32
@@ -177,3 +179,24 @@ def thresholds(d: int, nsub: int, dsub: int, queries: np.ndarray, model) -> np.n
     if rc != 0:
         raise ValueError(f"oracle_thresholds failed: {rc}")
     return out
+
+
+def entry_stats(index, queries: np.ndarray, neighbor_pos: np.ndarray):
+    """Entry usage and locality statistics of each query's neighbours (`neighbor_pos` [nq, k] int64
+    positions into the list-contiguous codes, -1 = none).  Returns (usage [nq, nsub] int32: distinct
+    entries used per subspace; rank_hist [nsub, ksub] int64: how often a neighbour's entry was the
+    r-th closest entry to the query's residual projection)."""
+    q = _c(queries, np.float32)
+    pos = _c(neighbor_pos, np.int64)
+    nq, k = pos.shape
+    cent = _c(index.coarse_centroids, np.float32)
+    cb = _c(index.codebooks, np.float32)
+    off = _c(index.list_offsets, np.int64)
+    codes = _c(index.codes, np.uint8)
+    usage = np.zeros((nq, index.nsub), np.int32)
+    hist = np.zeros((index.nsub, index.ksub), np.int64)
+    rc = _lib().oracle_entry_stats(index.d, index.nlist, index.nsub, index.dsub, index.ksub, _p(cent), _p(cb),
+                                   _p(off), _p(codes), _p(q), nq, _p(pos), k, _p(usage), _p(hist))
+    if rc != 0:
+        raise ValueError(f"oracle_entry_stats failed: {rc}")
+    return usage, hist

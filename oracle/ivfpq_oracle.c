@@ -15,7 +15,7 @@
  *   S2  selective L2-LUT: for every probed cluster the residual query - centroid;
  *       in every subspace the squared distance from the residual projection to each
  *       codebook entry; an entry is selected when that distance is within the
- *       threshold radius of the subspace (Sec. 2.1 steps B, C; Sec. 3.1 "Intuition of
+ *       threshold radius of the subspace (Sec. 2.1 steps B, C; Sec. 4.1 "Intuition of
  *       Algorithm Enhancement" and the last sentence of "Determining Proper
  *       Threshold"; Algorithm 2, whose ray test against a sphere of radius
  *       thres*thres_scale decides exactly d <= thres*thres_scale).  The table holds
@@ -24,12 +24,12 @@
  *   S3  distance calculation: every point of a probed cluster sums the table values
  *       of its codes over the subspaces in which its entry was selected (step D);
  *       each subspace whose entry was not selected contributes the large constant P
- *       instead of a table look-up (Sec. 4.3, paragraph after Algorithm 2).
+ *       instead of a table look-up (Sec. 5.3, paragraph after Algorithm 2).
  *   S4  the k smallest (distance, id) pairs, ascending (Sec. 2.1, last paragraph).
  * Dense search is the same with every entry selected.
  *
- * Hit-count scores (Sec. 4.4 "Aggressive Approximation: hit count-based Method"; the -L and -M
- * configurations of the evaluation plan in Sec. 5.1) replace S3's distance by a count, S1, S2's
+ * Hit-count scores (Sec. 5.4 "Aggressive Approximation: hit count-based Method"; the -L and -M
+ * configurations of the evaluation plan in Sec. 6.1) replace S3's distance by a count, S1, S2's
  * selection and S4 unchanged:
  *   score 1 (hit count): a point is ranked by the number of subspaces in which its entry was
  *       selected, more hits first.  Reported value: the number of subspaces missed (nsub - hits),
@@ -39,8 +39,8 @@
  *       one, 0 in between; more is better.  Reported value: nsub - score (0, 1 or 2 per subspace).
  *   The inner test is d2 <= 0.25f * (radius*scale)^2 on the same squared distance.
  *
- * Before S2, the query-specific thresholds can come from the dynamic threshold front-end (Sec. 3.1
- * "Determining Proper Threshold"; Algorithm 2, line 5): oracle_thresholds() below looks up the
+ * Before S2, the query-specific thresholds can come from the dynamic threshold front-end (Sec. 4.1
+ * "Determining Proper Threshold"; Algorithm 2, the threshold step): oracle_thresholds() below looks up the
  * density of the grid cell the query's projection falls into and evaluates the polynomial
  * regressor on it.
  *
@@ -282,10 +282,10 @@ int oracle_search(int d, int nlist, int nsub, int dsub, int ksub, const float* c
 }
 
 /*
- * Dynamic thresholds (Sec. 3.1 "Determining Proper Threshold": every 2-d subspace is divided into a
+ * Dynamic thresholds (Sec. 4.1 "Determining Proper Threshold": every 2-d subspace is divided into a
  * grid x grid map of cell densities; at search time the density of the cell that holds the query's
  * projection is read and a regression polynomial turns it into that query's threshold;
- * Algorithm 2, line 5: thres = poly_regressor(density_map(x, y)) with (x, y) the query's own
+ * Algorithm 2: thres = poly_regressor(density_map(x, y)) with (x, y) the query's own
  * projection, taken before the centroid is subtracted).
  *   density  [nsub][grid][grid]   row = cell index along the second coordinate, column = first
  *   origin   [nsub][2]            lower corner of the grid
@@ -319,4 +319,65 @@ int oracle_thresholds(int d, int nsub, int dsub, const float* queries, int64_t n
         }
     }
     return 0;
+}
+
+/*
+ * Entry usage and locality statistics of the neighbours of a query (Sec. 3.2 "Sparsity of Codebook
+ * Entries Used by Top-k Neighbors" and Sec. 3.3 "Spatial Locality of Codebook Entries Used by Top-k
+ * Neighbors").  For every query a list of neighbours is given as positions into the list-contiguous
+ * codes (-1 = none), normally its exact top-100.
+ *   usage[q][s]      number of distinct entries of codebook s that the neighbours of q are encoded
+ *                    with (the paper's usage ratio is this over ksub)
+ *   rank_hist[s][r]  += 1 for every (query, neighbour) whose entry in subspace s is the r-th closest
+ *                    entry (r = 0 closest) to the residual projection of the query against the
+ *                    centroid of the neighbour's list; entries are ordered by (squared distance,
+ *                    entry number).  Its running sum over r is the CDF of Sec. 3.3.
+ * rank_hist is accumulated into (the caller zeroes it); distances in the search's fp32 arithmetic.
+ */
+int oracle_entry_stats(int d, int nlist, int nsub, int dsub, int ksub, const float* cent, const float* codebooks,
+                       const int64_t* list_offsets, const uint8_t* codes, const float* queries, int64_t nq,
+                       const int64_t* neighbor_pos, int k, int32_t* usage, int64_t* rank_hist) {
+    if (d != nsub * dsub || ksub <= 0 || ksub > 256) return -2;
+    const int64_t ntotal = list_offsets[nlist];
+    float* dist = (float*)malloc(sizeof(float) * (size_t)ksub);
+    uint8_t* used = (uint8_t*)malloc((size_t)nsub * ksub);
+    int status = 0;
+    for (int64_t qi = 0; qi < nq; ++qi) {
+        const float* q = queries + qi * d;
+        memset(used, 0, (size_t)nsub * ksub);
+        for (int j = 0; j < k; ++j) {
+            const int64_t x = neighbor_pos[qi * k + j];
+            if (x < 0) continue;
+            if (x >= ntotal) { status = -3; continue; }
+            int c = 0;                                   /* the list that holds position x */
+            while (!(list_offsets[c] <= x && x < list_offsets[c + 1])) ++c;
+            for (int s = 0; s < nsub; ++s) {
+                const int own = codes[(size_t)x * nsub + s];
+                if (own >= ksub) { status = -3; continue; }
+                used[(size_t)s * ksub + own] = 1;
+                for (int e = 0; e < ksub; ++e) {
+                    const float* entry = codebooks + ((size_t)s * ksub + e) * dsub;
+                    float d2 = 0.0f;
+                    for (int t = 0; t < dsub; ++t) {
+                        float res = q[s * dsub + t] - cent[(size_t)c * d + s * dsub + t];
+                        float u = res - entry[t];
+                        d2 = fmaf(u, u, d2);
+                    }
+                    dist[e] = d2;
+                }
+                int rank = 0;
+                for (int e = 0; e < ksub; ++e)
+                    if (dist[e] < dist[own] || (dist[e] == dist[own] && e < own)) ++rank;
+                rank_hist[(size_t)s * ksub + rank] += 1;
+            }
+        }
+        for (int s = 0; s < nsub; ++s) {
+            int n = 0;
+            for (int e = 0; e < ksub; ++e) n += used[(size_t)s * ksub + e];
+            usage[qi * nsub + s] = n;
+        }
+    }
+    free(used);
+    free(dist);
+    return status;
 }

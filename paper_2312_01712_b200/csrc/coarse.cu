@@ -3,7 +3,7 @@
 //
 // The distance is evaluated in the direct form sum_j (q_j - c_j)^2 with one fused multiply-add
 // per dimension, j ascending, fp32: the selection must reproduce the defining arithmetic bit for
-// bit, and the GEMM form |c|^2 - 2 q.c + |q|^2 that the paper uses on tensor cores (Sec. 4.3,
+// bit, and the GEMM form |c|^2 - 2 q.c + |q|^2 that the paper uses on tensor cores (Sec. 5.3,
 // last paragraph) rounds differently near the nprobe-th distance.
 #include <mutex>
 

@@ -1,5 +1,5 @@
 // Filtering stage on the 5th-generation tensor cores (paper Sec. 2.1 "Online Search", step A; the
-// GEMM form |c|^2 - 2 q.c + |q|^2 of Sec. 4.3, last paragraph).
+// GEMM form |c|^2 - 2 q.c + |q|^2 of Sec. 5.3, last paragraph).
 //
 // The tensor cores only *propose*: the nprobe closest clusters are decided by the defining fp32
 // arithmetic (sum over dimensions of fma(t, t, acc), t = q_j - c_j, j ascending), because the probe

@@ -5,10 +5,10 @@
 //   1. forms the residual query - centroid (paper Sec. 2.1 "Online Search", step B);
 //   2. builds the look-up table in shared memory: thread e computes, per subspace, the squared
 //      distance between the residual projection and codebook entry e (step C) and keeps it only
-//      when it is within the squared threshold of that subspace (the selection of Sec. 3.1 /
+//      when it is within the squared threshold of that subspace (the selection of Sec. 4.1 /
 //      Algorithm 2, whose ray test decides exactly "distance <= thres * thres_scale");
-//      an unselected slot holds the miss constant P, so that the scan needs no branch for "the
-//      remaining search points [are] assigned with a large constant" (Sec. 4.3);
+//      an unselected slot holds the miss constant P, so that the scan needs no branch for the
+//      large constant that points with an unselected entry receive (Sec. 5.3);
 //   3. streams the cluster's codes (32-point interleaved blocks, one point per lane) and sums
 //      one table value per subspace (step D);
 //   4. feeds (distance, id) into a CTA-wide streaming top-k.

@@ -1,7 +1,7 @@
 // Persistent fused selective-LUT / list-scan / top-k kernel for the 16 x 8 product quantizer (16
 // subspaces of 8 dimensions, 256 entries), the shape of the SIFT-like workloads.  Same computation
-// as scan.cu (paper Sec. 2.1 steps B-D with the selection of Sec. 3.1 / Algorithm 2 and the miss
-// constant of Sec. 4.3).  One CTA per SM loops over (query, probe slice) items.
+// as scan.cu (paper Sec. 2.1 steps B-D with the selection of Sec. 4.1 / Algorithm 2 and the miss
+// constant of Sec. 5.3).  One CTA per SM loops over (query, probe slice) items.
 //
 //   * Two instances, chosen when the index is loaded.  16 warps (128 registers per thread): the
 //     whole 128 KB codebook lives in registers - thread t owns subspace c = t & 15 and the entries

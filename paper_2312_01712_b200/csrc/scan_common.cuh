@@ -40,7 +40,7 @@ struct ScanParams {
 
 // What a table slot holds for an entry at squared distance d2 from the residual projection, given
 // whether it was selected (`hit`: d2 <= thr, always true for the dense search).  Distances: the
-// squared distance, or the miss constant P (paper Sec. 4.3).  Count scores (Sec. 4.4): 0 / 1 for
+// squared distance, or the miss constant P (paper Sec. 5.3).  Count scores (Sec. 5.4): 0 / 1 for
 // selected / not selected; with the inner sphere of half the radius 0 / 1 / 2 for inside the inner
 // sphere / between the two / outside both.  The list scan sums slots, whatever they hold.
 __device__ __forceinline__ float table_value(int score, bool hit, float d2, float thr, float P) {

@@ -1,7 +1,7 @@
 // Rotated-layout variant of the fused selective-LUT / list-scan / top-k kernel.
 //
-// Same computation as scan.cu (paper Sec. 2.1 steps B-D with the selection of Sec. 3.1 /
-// Algorithm 2 and the miss constant of Sec. 4.3), different shared-memory organisation, chosen
+// Same computation as scan.cu (paper Sec. 2.1 steps B-D with the selection of Sec. 4.1 /
+// Algorithm 2 and the miss constant of Sec. 5.3), different shared-memory organisation, chosen
 // so that the table gathers of a warp never collide on a bank whatever the codes are:
 //
 //   * the subspaces are split into groups of width w (a power of two, 32 or less); a group's table

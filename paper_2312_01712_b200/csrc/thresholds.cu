@@ -1,4 +1,4 @@
-// Dynamic threshold front-end (paper Sec. 3.1 "Determining Proper Threshold"; Algorithm 2, line 5:
+// Dynamic threshold front-end (paper Sec. 4.1 "Determining Proper Threshold"; Algorithm 2:
 // thres = poly_regressor(density_map(x, y))).  Every 2-d subspace carries a grid x grid map of
 // cell densities; the threshold of a query in a subspace is a polynomial of the density of the cell
 // that the query's own projection (before the centroid is subtracted) falls into.  The output is

@@ -1,4 +1,4 @@
-"""GPU parity of the hit-count scores (paper Sec. 4.4 "Aggressive Approximation: hit count-based
+"""GPU parity of the hit-count scores (paper Sec. 5.4 "Aggressive Approximation: hit count-based
 Method") against the CPU oracle.  The reported values are small integers and ties are decided by
 id on both sides, so values and id lists must be identical, not merely within a tolerance."""
 

@@ -1,5 +1,5 @@
-"""GPU parity of the dynamic threshold front-end (paper Sec. 3.1 "Determining Proper Threshold";
-Algorithm 2, line 5) against the CPU oracle: thresholds are fp32 results of a table look-up and a
+"""GPU parity of the dynamic threshold front-end (paper Sec. 4.1 "Determining Proper Threshold";
+Algorithm 2, the threshold step) against the CPU oracle: thresholds are fp32 results of a table look-up and a
 fixed-order Horner evaluation, so the comparison is bit for bit."""
 
 import numpy as np

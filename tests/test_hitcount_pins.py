@@ -1,4 +1,4 @@
-"""Pins for the hit-count scores of the CPU oracle (paper Sec. 4.4 "Aggressive Approximation: hit
+"""Pins for the hit-count scores of the CPU oracle (paper Sec. 5.4 "Aggressive Approximation: hit
 count-based Method"): values worked by hand, limits in which the score is known in closed form, and
 identities that tie the counts to the distance mode, which has pins of its own."""
 
@@ -93,7 +93,7 @@ def test_top_k_is_the_sorted_prefix_of_all_visited_points(wl_pq2, score):
 
 
 def test_more_hits_means_closer_on_average(wl_small):
-    """The observation the method rests on (Sec. 4.4): the hit count correlates with the distance.
+    """The observation the method rests on (Sec. 5.4): the hit count correlates with the distance.
     On the synthetic mixture the points ranked first by hit count are closer (dense ADC distance)
     than the visited points on average, and the reward/penalty score ranks at least as well."""
     idx, q = wl_small.index, wl_small.queries[:48]
