@@ -140,6 +140,27 @@ typedef struct {
 int ivfpq_query_thresholds(const ivfpq_index_t* index, const float* queries, int64_t nq,
                            const ivfpq_threshold_model_t* model, float* radius_out, void* stream);
 
+/* Entry usage and locality statistics of each query's neighbours (Sec. 3.2 "Sparsity of Codebook
+ * Entries Used by Top-k Neighbors", Sec. 3.3 "Spatial Locality of Codebook Entries Used by Top-k
+ * Neighbors"); an analysis tool for choosing radii, not a step of the search.
+ *   codes         dev [ntotal][nsub]: the list-contiguous codes the index was loaded from (the
+ *                 handle keeps only a re-laid-out copy)
+ *   neighbor_pos  dev [nq][k]: positions into `codes` of each query's neighbours (normally its
+ *                 exact top-100), -1 = none; 1 <= k <= IVFPQ_MAX_K
+ *   usage_out     dev [nq][nsub]: distinct entries of codebook s among the query's neighbours (the
+ *                 paper's usage ratio is this / ksub)
+ *   rank_hist     dev [nsub][ksub] unsigned 64-bit, ACCUMULATED into (zero it first): one count per
+ *                 (query, neighbour, subspace) at r = the number of entries ordered before the
+ *                 neighbour's own entry by (squared distance to the query's residual projection
+ *                 against the centroid of the neighbour's list, entry number); the running sum
+ *                 over r is the CDF of Sec. 3.3.  Distances in the search's fp32 arithmetic.
+ *   flags         dev, one int32, OR-ed into (zero it first): non-zero afterwards when a position
+ *                 >= ntotal or a code >= ksub was met (that neighbour or subspace was skipped).
+ * Asynchronous on `stream`; allocates nothing. */
+int ivfpq_entry_stats(const ivfpq_index_t* index, const uint8_t* codes, const float* queries, int64_t nq,
+                      const int64_t* neighbor_pos, int32_t k, int32_t* usage_out,
+                      unsigned long long* rank_hist, int32_t* flags, void* stream);
+
 /* Workspace (dev, 256-byte aligned) needed by one search call of this shape. */
 size_t ivfpq_search_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k);
 

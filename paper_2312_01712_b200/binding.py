@@ -39,6 +39,7 @@ EXPORTS = (
     "ivfpq_search_host_workspace_bytes", "ivfpq_search_host", "ivfpq_sync_status",
     "ivfpq_index_set_option", "ivfpq_last_launch_count", "ivfpq_last_stage_ms", "ivfpq_error_string",
     "ivfpq_debug_probes", "ivfpq_debug_search", "ivfpq_probe_static", "ivfpq_query_thresholds",
+    "ivfpq_entry_stats",
 )
 
 
@@ -112,6 +113,8 @@ def load_library() -> ctypes.CDLL:
     lib.ivfpq_debug_search.restype = ctypes.c_int
     lib.ivfpq_query_thresholds.argtypes = [vp, vp, i64, ctypes.POINTER(ivfpq_threshold_model_t), vp, vp]
     lib.ivfpq_query_thresholds.restype = ctypes.c_int
+    lib.ivfpq_entry_stats.argtypes = [vp, vp, vp, i64, vp, i32, vp, vp, vp, vp]
+    lib.ivfpq_entry_stats.restype = ctypes.c_int
     lib.ivfpq_probe_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
     lib.ivfpq_probe_static.restype = ctypes.c_int
     _lib = lib
@@ -380,3 +383,27 @@ def ivfpq_query_thresholds(ix: IndexHandle, queries: torch.Tensor, model: Thresh
     _check(load_library().ivfpq_query_thresholds(ix.handle, queries.data_ptr(), nq, ctypes.byref(model.struct),
                                                  out.data_ptr(), _stream()), "ivfpq_query_thresholds")
     return out
+
+
+def ivfpq_entry_stats(ix: IndexHandle, codes: torch.Tensor, queries: torch.Tensor, neighbor_pos: torch.Tensor,
+                      rank_hist: Optional[torch.Tensor] = None):
+    """Entry usage and locality statistics of each query's neighbours.  `codes` [ntotal, nsub] uint8
+    (list-contiguous, on the device), `neighbor_pos` [nq, k] int64 positions into it (-1 = none).
+    Returns (usage [nq, nsub] int32, rank_hist [nsub, ksub] int64, accumulated into when given,
+    flags: non-zero when an out-of-range position or code was skipped)."""
+    nq, k = neighbor_pos.shape
+    if codes.dtype != torch.uint8 or not codes.is_cuda or not codes.is_contiguous() or tuple(codes.shape) != (ix.ntotal, ix.nsub):
+        raise ValueError("codes must be a contiguous uint8 CUDA tensor [ntotal, nsub]")
+    if neighbor_pos.dtype != torch.int64 or not neighbor_pos.is_cuda or not neighbor_pos.is_contiguous():
+        raise ValueError("neighbor_pos must be a contiguous int64 CUDA tensor [nq, k]")
+    if queries.dtype != torch.float32 or not queries.is_cuda or not queries.is_contiguous() or tuple(queries.shape) != (nq, ix.d):
+        raise ValueError("queries must be a contiguous fp32 CUDA tensor [nq, d]")
+    dev = queries.device
+    usage = torch.empty((nq, ix.nsub), dtype=torch.int32, device=dev)
+    if rank_hist is None:
+        rank_hist = torch.zeros((ix.nsub, ix.ksub), dtype=torch.int64, device=dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    _check(load_library().ivfpq_entry_stats(ix.handle, codes.data_ptr(), queries.data_ptr(), nq, neighbor_pos.data_ptr(),
+                                            k, usage.data_ptr(), rank_hist.data_ptr(), flags.data_ptr(), _stream()),
+           "ivfpq_entry_stats")
+    return usage, rank_hist, int(flags.item())

@@ -278,6 +278,19 @@ int ivfpq_query_thresholds(const ivfpq_index_t* index, const float* queries, int
     return IVFPQ_OK;
 }
 
+int ivfpq_entry_stats(const ivfpq_index_t* index, const uint8_t* codes, const float* queries, int64_t nq,
+                      const int64_t* neighbor_pos, int32_t k, int32_t* usage_out,
+                      unsigned long long* rank_hist, int32_t* flags, void* stream) {
+    if (!index || !codes || !queries || !neighbor_pos || !usage_out || !rank_hist || !flags)
+        return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (nq <= 0 || k <= 0) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (k > IVFPQ_MAX_K || nq > (int64_t)1 << 30) return IVFPQ_ERR_UNSUPPORTED;
+    if (launch_entry_stats(index, codes, queries, nq, neighbor_pos, k, usage_out, rank_hist, flags,
+                           reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    return IVFPQ_OK;
+}
+
 size_t ivfpq_search_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k) {
     if (check_search_shape(index, nq, nprobe, k) != IVFPQ_OK) return 0;
     return plan_workspace(index, nq, nprobe, k).total;

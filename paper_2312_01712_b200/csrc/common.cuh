@@ -116,6 +116,9 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
 cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,
                           float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
                           int* status, cudaStream_t st, int64_t* launches);
+cudaError_t launch_entry_stats(const ivfpq_index* ix, const uint8_t* codes, const float* queries, int64_t nq,
+                               const int64_t* nbr, int k, int32_t* usage, unsigned long long* rank_hist, int* status,
+                               cudaStream_t st);
 cudaError_t launch_thresholds(const float* queries, int64_t nq, int nsub, const ivfpq_threshold_model_t* m,
                               float* radius, cudaStream_t st);
 cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws, cudaStream_t st,
