@@ -71,6 +71,8 @@ def _lib() -> ctypes.CDLL:
         lib.oracle_search_scored.restype = i32
         lib.oracle_entry_stats.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i64, vp, i32, vp, vp]
         lib.oracle_entry_stats.restype = i32
+        lib.oracle_search_ip.argtypes = list(lib.oracle_search.argtypes)
+        lib.oracle_search_ip.restype = i32
         lib.oracle_thresholds.argtypes = [i32, i32, i32, vp, i64, i32, i32, vp, vp, vp, vp, vp]
         lib.oracle_thresholds.restype = i32
         lib.oracle_num_threads.restype = i32
@@ -110,7 +112,7 @@ def coarse(index, queries: np.ndarray, nprobe: int):
 
 def search(index, queries: np.ndarray, nprobe: int, k: int, *, dense: bool = False,
            radius: Optional[np.ndarray] = None, scale: float = 1.0, miss_penalty: float = -1.0,
-           dumps: bool = False, visit_stride: int = 0, score: int = 0) -> dict:
+           dumps: bool = False, visit_stride: int = 0, score: int = 0, metric: Optional[int] = None) -> dict:
     """Dense (`dense=True`) or sparsity-aware search.  `radius` is [nsub] (one
     threshold per subspace) or [nq, nsub] (per query and subspace).  Returns a dict
     with `dist` [nq, k] fp32 and `ids` [nq, k] int32; with `dumps=True` also
@@ -118,7 +120,9 @@ def search(index, queries: np.ndarray, nprobe: int, k: int, *, dense: bool = Fal
     with `visit_stride > 0` also per-visited-point `visit_hits` (uint64 bit sets),
     `visit_dist` and `visit_ids`, each [nq, visit_stride] in visiting order.
     `score`: 0 = distances; 1 = hit count (reported value: subspaces missed); 2 = reward/penalty
-    with an inner sphere of half the radius (reported value: nsub - score)."""
+    with an inner sphere of half the radius (reported value: nsub - score).
+    `metric` (default: the index's): 0 = squared L2; 1 = inner product, where `dist`, `probe_d`
+    and `visit_dist` hold similarities, larger first, padded with -inf."""
     q = _c(queries, np.float32)
     nq = q.shape[0]
     cent = _c(index.coarse_centroids, np.float32)
@@ -152,6 +156,22 @@ def search(index, queries: np.ndarray, nprobe: int, k: int, *, dense: bool = Fal
         vd = np.full((nq, visit_stride), np.inf, np.float32)
         vi = np.full((nq, visit_stride), -1, np.int32)
         res.update(visit_hits=vh, visit_dist=vd, visit_ids=vi)
+    metric = int(getattr(index, "metric", 0)) if metric is None else int(metric)
+    if metric == 1:
+        if score != 0:
+            raise ValueError("the count scores are defined for the L2 metric only")
+        if visit_stride > 0:
+            vd.fill(-np.inf)
+        rc = _lib().oracle_search_ip(index.d, index.nlist, index.nsub, index.dsub, index.ksub,
+                                     _p(cent), _p(cb), _p(off), _p(codes), _p(ids),
+                                     _p(q), nq, nprobe, 1 if dense else 0,
+                                     _p(rad), mode, float(scale), float(miss_penalty), k,
+                                     _p(out_d), _p(out_i),
+                                     _p(pid), _p(pd), _p(masks), _p(vcount), int(visit_stride),
+                                     _p(vh), _p(vd), _p(vi))
+        if rc != 0:
+            raise ValueError(f"oracle_search_ip failed: {rc}")
+        return res
     rc = _lib().oracle_search_scored(index.d, index.nlist, index.nsub, index.dsub, index.ksub,
                                      _p(cent), _p(cb), _p(off), _p(codes), _p(ids),
                                      _p(q), nq, nprobe, 1 if dense else 0,

@@ -39,6 +39,18 @@
  *       one, 0 in between; more is better.  Reported value: nsub - score (0, 1 or 2 per subspace).
  *   The inner test is d2 <= 0.25f * (radius*scale)^2 on the same squared distance.
  *
+ * Inner-product similarity (Sec. 4.2 "Inner Product Similarity Support"): oracle_search_ip() below.
+ *   S1  filtering by inner product: the nprobe clusters with the largest q.c.
+ *   S2  the sphere of entry e gets the radius sqrt(R^2 + |e|^2), R the subspace's threshold: the
+ *       entry is selected when |q_s - e|^2 <= R^2 + |e|^2, and its table value is the inner product
+ *       q_s.e, which the paper recovers from the hit time as (|q_s|^2 + |e|^2 - |q_s - e|^2) / 2.
+ *       The projection is the query's own: with residual codes x ~ c + sum_s e_s the similarity
+ *       splits into q.c (known from S1) plus q_s.e_s per subspace, so the table does not depend
+ *       on the cluster.
+ *   S3  similarity = q.c + sum of the table values of the selected subspaces - m * P for the m
+ *       subspaces whose entry was not selected (the large constant, now a penalty).
+ *   S4  the k largest (similarity, then smaller id), padded with (-inf, -1).
+ *
  * Before S2, the query-specific thresholds can come from the dynamic threshold front-end (Sec. 4.1
  * "Determining Proper Threshold"; Algorithm 2, the threshold step): oracle_thresholds() below looks up the
  * density of the grid cell the query's projection falls into and evaluates the polynomial
@@ -380,4 +392,151 @@ int oracle_entry_stats(int d, int nlist, int nsub, int dsub, int ksub, const flo
     free(used);
     free(dist);
     return status;
+}
+
+/* cand_less for similarities: larger first, then smaller id */
+static int cand_greater(const void* a, const void* b) {
+    const cand_t* x = (const cand_t*)a;
+    const cand_t* y = (const cand_t*)b;
+    if (x->dist > y->dist) return -1;
+    if (x->dist < y->dist) return 1;
+    if (x->id < y->id) return -1;
+    if (x->id > y->id) return 1;
+    return 0;
+}
+
+static float dot_f32(const float* a, const float* b, int n) {
+    float acc = 0.0f;
+    for (int j = 0; j < n; ++j) acc = fmaf(a[j], b[j], acc);
+    return acc;
+}
+
+/*
+ * Search under the inner-product similarity (header comment; Sec. 4.2 "Inner Product Similarity
+ * Support").  Arguments as oracle_search; probe_d and visit_dist hold similarities; dense != 0
+ * selects every entry.  miss_penalty < 0 asks for the default P = sum over subspaces of
+ * (radius*scale)^2.
+ */
+int oracle_search_ip(int d, int nlist, int nsub, int dsub, int ksub, const float* cent,
+                     const float* codebooks, const int64_t* list_offsets, const uint8_t* codes,
+                     const int32_t* ids, const float* queries, int64_t nq, int nprobe, int dense,
+                     const float* radius, int radius_mode, float scale, float miss_penalty, int k,
+                     float* out_sim, int32_t* out_ids, int32_t* probe_ids_out, float* probe_ip_out,
+                     uint32_t* masks_out, int64_t* visit_count, int64_t visit_stride,
+                     uint64_t* visit_hits, float* visit_sim, int32_t* visit_ids) {
+    if (d != nsub * dsub || ksub <= 0 || ksub > 256 || nsub > 64) return -2;
+    if (nprobe <= 0 || nprobe > nlist || k <= 0) return -1;
+    if (!dense && radius == NULL) return -1;
+
+#pragma omp parallel
+    {
+        cand_t* scratch = (cand_t*)malloc(sizeof(cand_t) * (size_t)nlist);
+        float* lut = (float*)malloc(sizeof(float) * (size_t)nsub * ksub);
+        uint8_t* hit = (uint8_t*)malloc((size_t)nsub * ksub);
+        float* r2 = (float*)malloc(sizeof(float) * (size_t)nsub);
+        size_t cap = 1024, n = 0;
+        cand_t* vis = (cand_t*)malloc(sizeof(cand_t) * cap);
+
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t qi = 0; qi < nq; ++qi) {
+            const float* q = queries + qi * d;
+            /* S1: the nprobe largest inner products, ties to the smaller cluster id */
+            for (int c = 0; c < nlist; ++c) {
+                scratch[c].dist = dot_f32(q, cent + (size_t)c * d, d);
+                scratch[c].id = c;
+            }
+            qsort(scratch, (size_t)nlist, sizeof(cand_t), cand_greater);
+            if (probe_ids_out)
+                for (int p = 0; p < nprobe; ++p) probe_ids_out[qi * nprobe + p] = scratch[p].id;
+            if (probe_ip_out)
+                for (int p = 0; p < nprobe; ++p) probe_ip_out[qi * nprobe + p] = scratch[p].dist;
+
+            float P = 0.0f;
+            if (!dense) {
+                const float* rad = radius_mode == 1 ? radius + qi * nsub : radius;
+                float acc = 0.0f;
+                for (int s = 0; s < nsub; ++s) {
+                    float r = rad[s] * scale;
+                    r2[s] = r * r;
+                    acc = acc + r2[s];
+                }
+                P = miss_penalty >= 0.0f ? miss_penalty : acc;
+            }
+
+            /* S2: one table per query */
+            for (int s = 0; s < nsub; ++s) {
+                uint32_t mrow[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+                for (int e = 0; e < ksub; ++e) {
+                    const float* entry = codebooks + ((size_t)s * ksub + e) * dsub;
+                    float d2 = 0.0f;
+                    for (int j = 0; j < dsub; ++j) {
+                        float t = q[s * dsub + j] - entry[j];
+                        d2 = fmaf(t, t, d2);
+                    }
+                    float en2 = dot_f32(entry, entry, dsub);
+                    int h = dense ? 1 : (d2 <= r2[s] + en2);
+                    lut[(size_t)s * ksub + e] = dot_f32(q + s * dsub, entry, dsub);
+                    hit[(size_t)s * ksub + e] = (uint8_t)h;
+                    if (h) mrow[e >> 5] |= 1u << (e & 31);
+                }
+                if (masks_out)
+                    for (int p = 0; p < nprobe; ++p)
+                        memcpy(masks_out + (((size_t)qi * nprobe + p) * nsub + s) * 8, mrow, sizeof(mrow));
+            }
+
+            n = 0;
+            int64_t nvis = 0;
+            for (int p = 0; p < nprobe; ++p) {
+                const int c = scratch[p].id;
+                const float base = scratch[p].dist; /* q.c */
+                for (int64_t x = list_offsets[c]; x < list_offsets[c + 1]; ++x) {
+                    const uint8_t* code = codes + (size_t)x * nsub;
+                    float S = base;
+                    int m = 0;
+                    uint64_t hs = 0;
+                    for (int s = 0; s < nsub; ++s) {
+                        int e = code[s];
+                        if (e < ksub && hit[(size_t)s * ksub + e]) {
+                            S = S + lut[(size_t)s * ksub + e];
+                            hs |= (uint64_t)1 << s;
+                        } else {
+                            m += 1;
+                        }
+                    }
+                    float sim = (m == 0) ? S : fmaf(-(float)m, P, S);
+                    if (n == cap) {
+                        cap *= 2;
+                        vis = (cand_t*)realloc(vis, sizeof(cand_t) * cap);
+                    }
+                    vis[n].dist = sim;
+                    vis[n].id = ids[x];
+                    ++n;
+                    if (nvis < visit_stride) {
+                        if (visit_hits) visit_hits[qi * visit_stride + nvis] = hs;
+                        if (visit_sim) visit_sim[qi * visit_stride + nvis] = sim;
+                        if (visit_ids) visit_ids[qi * visit_stride + nvis] = ids[x];
+                    }
+                    ++nvis;
+                }
+            }
+            if (visit_count) visit_count[qi] = nvis;
+
+            qsort(vis, n, sizeof(cand_t), cand_greater);
+            for (int i = 0; i < k; ++i) {
+                if ((size_t)i < n) {
+                    out_sim[qi * k + i] = vis[i].dist;
+                    out_ids[qi * k + i] = vis[i].id;
+                } else {
+                    out_sim[qi * k + i] = -INFINITY;
+                    out_ids[qi * k + i] = -1;
+                }
+            }
+        }
+        free(vis);
+        free(r2);
+        free(hit);
+        free(lut);
+        free(scratch);
+    }
+    return 0;
 }
