@@ -19,6 +19,22 @@
  * nlist = IVF clusters (C), nprobe = probed clusters per query (nprobs).
  * All distances are SQUARED L2 (Eq. "metric").  All floating point is fp32.
  *
+ * Inner-product similarity (metric = IVFPQ_METRIC_IP; Sec. 4.2 "Inner Product Similarity Support"):
+ *   (1) filtering keeps the nprobe clusters with the LARGEST inner product q.c;
+ *   (2) the table is built from the query's own projection q_s (with residual codes the similarity
+ *       splits into q.c plus q_s.e per subspace, so one table serves all probed clusters); the
+ *       sphere of entry e has radius sqrt(R^2 + |e|^2), R the subspace's threshold: the entry is
+ *       selected when |q_s - e|^2 <= R^2 + |e|^2, and its table value is q_s.e (the paper recovers
+ *       it from the hit time as (|q_s|^2 + |e|^2 - |q_s - e|^2) / 2);
+ *   (3) similarity = q.c + sum of the selected table values - m * P for m unselected subspaces
+ *       (miss_penalty P, default sum of (radius*scale)^2); the k LARGEST (similarity, then smaller
+ *       id) per query, padded with (-inf, -1).
+ *   out_dist, probe_d and the dumps then hold similarities.  Defining arithmetic: inner products
+ *   and |e|^2 as one fused multiply-add per dimension, ascending; |q_s - e|^2 as for L2; the test
+ *   compares with the fp32 sum R^2 + |e|^2.  The count scores, ivfpq_probe_static and the
+ *   specialised scan kernels are L2-only: an inner-product index is served by the exact SIMT
+ *   filtering kernels and the generic scan kernel.
+ *
  * Conventions for every entry point:
  *   - returns IVFPQ_OK (0) or a negative IVFPQ_ERR_* code; never throws, never aborts;
  *   - "dev" pointers are device memory owned by the caller (e.g. torch tensors) that must stay
@@ -47,6 +63,8 @@ extern "C" {
 #define IVFPQ_ERR_DEVICE_FLAG (-5)      /* a kernel raised its bounds / bounded-wait error flag   */
 #define IVFPQ_ERR_STATIC_LIMIT (-6)     /* index too large for the scratch built into the library */
 
+#define IVFPQ_METRIC_L2 0
+#define IVFPQ_METRIC_IP 1
 #define IVFPQ_MAX_K 1024
 #define IVFPQ_MAX_NPROBE 1024
 #define IVFPQ_MAX_NSUB 64
@@ -62,7 +80,7 @@ typedef struct {
     int32_t nsub;   /* PQ subspaces, 1..64                                               */
     int32_t dsub;   /* dimensions per subspace, 1..16                                    */
     int32_t ksub;   /* entries per codebook, 1..256                                      */
-    int32_t metric; /* 0 = squared L2 (the only one supported)                           */
+    int32_t metric; /* IVFPQ_METRIC_L2 (squared L2) or IVFPQ_METRIC_IP (inner product)    */
     int64_t ntotal; /* encoded points                                                    */
     const float* coarse_centroids; /* dev  [nlist][d]                                    */
     const float* codebooks;        /* dev  [nsub][ksub][dsub], trained on residuals      */

@@ -29,6 +29,8 @@ IVFPQ_STATIC_SCRATCH_BYTES = 8 << 20
 IVFPQ_STATIC_MAX_NLIST = 16384
 IVFPQ_OPT_NSPLIT = 1
 IVFPQ_OPT_TIMING = 2
+IVFPQ_METRIC_L2 = 0
+IVFPQ_METRIC_IP = 1
 IVFPQ_SCORE_DISTANCE = 0
 IVFPQ_SCORE_HIT_COUNT = 1
 IVFPQ_SCORE_REWARD_PENALTY = 2
@@ -176,7 +178,8 @@ def ivfpq_index_load(index, device="cuda") -> IndexHandle:
     codes = torch.from_numpy(np.ascontiguousarray(index.codes, np.uint8)).to(dev)
     ids = torch.from_numpy(np.ascontiguousarray(index.ids, np.int32)).to(dev)
     off = np.ascontiguousarray(index.list_offsets, np.int64)
-    desc = ivfpq_index_desc_t(index.d, index.nlist, index.nsub, index.dsub, index.ksub, 0, index.ntotal,
+    metric = int(getattr(index, "metric", IVFPQ_METRIC_L2))
+    desc = ivfpq_index_desc_t(index.d, index.nlist, index.nsub, index.dsub, index.ksub, metric, index.ntotal,
                               cent.data_ptr(), cb.data_ptr(), off.ctypes.data, codes.data_ptr(), ids.data_ptr())
     nbytes = lib.ivfpq_index_derived_bytes(ctypes.byref(desc))
     if nbytes == 0:
@@ -188,7 +191,7 @@ def ivfpq_index_load(index, device="cuda") -> IndexHandle:
                "ivfpq_index_load")
         torch.cuda.current_stream().synchronize()   # the source codes may be released now
     meta = dict(d=index.d, nlist=index.nlist, nsub=index.nsub, dsub=index.dsub, ksub=index.ksub,
-                ntotal=index.ntotal)
+                ntotal=index.ntotal, metric=metric)
     return IndexHandle(handle.value, {"cent": cent, "cb": cb, "ids": ids, "derived": derived}, meta)
 
 

@@ -27,7 +27,7 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     if (d->d <= 0 || d->nlist <= 0 || d->nsub <= 0 || d->dsub <= 0 || d->ksub <= 0 || d->ntotal < 0)
         return IVFPQ_ERR_INVALID_ARGUMENT;
     if ((int64_t)d->nsub * d->dsub != d->d) return IVFPQ_ERR_INVALID_ARGUMENT;
-    if (d->metric != 0 || d->ksub > 256 || d->nsub > IVFPQ_MAX_NSUB || d->dsub > IVFPQ_MAX_DSUB)
+    if ((d->metric != IVFPQ_METRIC_L2 && d->metric != IVFPQ_METRIC_IP) || d->ksub > 256 || d->nsub > IVFPQ_MAX_NSUB || d->dsub > IVFPQ_MAX_DSUB)
         return IVFPQ_ERR_UNSUPPORTED;
     if (d->ntotal > 0x7FFFFFFFll) return IVFPQ_ERR_UNSUPPORTED;  // ids are int32
     if (!d->list_offsets) return IVFPQ_ERR_INVALID_ARGUMENT;
@@ -49,13 +49,14 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     out->list_blk_off = off;
     off = align_up(off + sizeof(int64_t) * (size_t)(d->nlist + 1), 256);
     out->codes_off = off;
-    out->rot = (rot_supported(d->nsub, d->dsub) && rot_group_widths(d->nsub, out->gw)) ? 1 : 0;
+    // the rotated layouts belong to the L2-only kernels
+    out->rot = (d->metric == IVFPQ_METRIC_L2 && rot_supported(d->nsub, d->dsub) && rot_group_widths(d->nsub, out->gw)) ? 1 : 0;
     out->block_bytes = out->rot ? rot_block_bytes(out->gw) : kPointsPerBlock * out->nw * 4;
     off = align_up(off + (size_t)nblocks * out->block_bytes, 256);
     out->cbt_off = off;
     if (out->rot) off = align_up(off + (size_t)d->nsub * 256 * d->dsub * 4, 256);
     out->cnorm_off = off;
-    out->mma = coarse_mma_supported(d->d, d->nlist) ? 1 : 0;
+    out->mma = (d->metric == IVFPQ_METRIC_L2 && coarse_mma_supported(d->d, d->nlist)) ? 1 : 0;
     if (out->mma) off = align_up(off + coarse_mma_derived_bytes(d->nlist), 256);
     out->total = off > 0 ? off : 256;
     return IVFPQ_OK;
@@ -79,6 +80,7 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
         if (!a.radius || (a.radius_mode != 0 && a.radius_mode != 1)) return IVFPQ_ERR_INVALID_ARGUMENT;
         if (isnan(a.scale) || isnan(a.miss_penalty)) return IVFPQ_ERR_INVALID_ARGUMENT;
         if (a.score < IVFPQ_SCORE_DISTANCE || a.score > IVFPQ_SCORE_REWARD_PENALTY) return IVFPQ_ERR_INVALID_ARGUMENT;
+        if (a.score != IVFPQ_SCORE_DISTANCE && ix->metric != IVFPQ_METRIC_L2) return IVFPQ_ERR_UNSUPPORTED;
     }
     if (!aligned(a.queries, 4) || !aligned(workspace, 256)) return IVFPQ_ERR_WORKSPACE;
     if (!probes_only && !aligned(a.queries, 16)) return IVFPQ_ERR_INVALID_ARGUMENT;  // the scan kernels load rows as float4
@@ -106,8 +108,12 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
     if (a.probe_ids_out &&
         cudaMemcpyAsync(a.probe_ids_out, probe_ids, pbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return IVFPQ_ERR_CUDA;
-    if (a.probe_d_out && cudaMemcpyAsync(a.probe_d_out, probe_d, pbytes, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-        return IVFPQ_ERR_CUDA;
+    if (a.probe_d_out) {
+        const cudaError_t e = ix->metric == IVFPQ_METRIC_IP
+                                  ? launch_negate(probe_d, a.probe_d_out, (int64_t)a.nq * a.nprobe, st)
+                                  : cudaMemcpyAsync(a.probe_d_out, probe_d, pbytes, cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return IVFPQ_ERR_CUDA;
+    }
     if (!probes_only) {
         if (launch_scan(a, wl, ws, st, &launches) != cudaSuccess) return IVFPQ_ERR_CUDA;
     }
@@ -193,6 +199,7 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->dsub = desc->dsub;
     ix->ksub = desc->ksub;
     ix->ntotal = desc->ntotal;
+    ix->metric = desc->metric;
     ix->cent = desc->coarse_centroids;
     ix->cb = desc->codebooks;
     ix->ids = desc->ids;

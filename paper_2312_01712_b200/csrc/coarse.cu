@@ -18,7 +18,10 @@ constexpr int TQ = 64;   // queries per CTA tile
 constexpr int TC = 64;   // centroids per CTA tile
 constexpr int TK = 16;   // dimensions per shared-memory stage
 
-// out[(q - q0) * nlist + c] = sum_j fma(q_j - c_j, q_j - c_j, acc), for q in [q0, q0 + nqc)
+// out[(q - q0) * nlist + c] = sum_j fma(q_j - c_j, q_j - c_j, acc), for q in [q0, q0 + nqc).
+// IP (paper Sec. 4.2 "Inner Product Similarity Support": filtering by inner product): the tile holds
+// -(sum_j fma(q_j, c_j, acc)), so that "smallest first" selects the largest inner products.
+template <bool IP>
 __global__ void __launch_bounds__(256) coarse_dist_kernel(const float* __restrict__ queries, int64_t q0,
                                                           int nqc, const float* __restrict__ cent,
                                                           int nlist, int d, float* __restrict__ out) {
@@ -59,8 +62,12 @@ __global__ void __launch_bounds__(256) coarse_dist_kernel(const float* __restric
             for (int a = 0; a < 4; ++a)
 #pragma unroll
                 for (int b = 0; b < 4; ++b) {
-                    float t = __fsub_rn(qa[a], ca[b]);
-                    acc[a][b] = __fmaf_rn(t, t, acc[a][b]);
+                    if (IP) {
+                        acc[a][b] = __fmaf_rn(qa[a], ca[b], acc[a][b]);
+                    } else {
+                        float t = __fsub_rn(qa[a], ca[b]);
+                        acc[a][b] = __fmaf_rn(t, t, acc[a][b]);
+                    }
                 }
         }
     }
@@ -71,12 +78,14 @@ __global__ void __launch_bounds__(256) coarse_dist_kernel(const float* __restric
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
             int c = cbase + tx * 4 + b;
-            if (c < nlist) out[(int64_t)q * nlist + c] = acc[a][b];
+            if (c < nlist) out[(int64_t)q * nlist + c] = IP ? -acc[a][b] : acc[a][b];
         }
     }
 }
 
-// One CTA per query: the nprobe smallest (distance, cluster id) pairs, ascending.
+// One CTA per query: the nprobe smallest (distance, cluster id) pairs, ascending.  SIGNED: the
+// values may be negative (negated inner products) and the keys use the order-preserving bit map.
+template <bool SIGNED>
 __global__ void __launch_bounds__(256) select_probes_kernel(const float* __restrict__ dist, int nlist,
                                                             int nprobe, int32_t* __restrict__ probe_ids,
                                                             float* __restrict__ probe_d, int64_t q0,
@@ -85,13 +94,14 @@ __global__ void __launch_bounds__(256) select_probes_kernel(const float* __restr
     __shared__ int cnt;
     __shared__ unsigned long long tau;
     __shared__ int hist[kTopkHistInts];
-    TopkState t{buf, &cnt, &tau, hist};
+    TopkState t{buf, &cnt, &tau, hist, SIGNED ? kKeyPadSigned : kKeyPad};
     topk_init(t);
     const float* row = dist + (int64_t)blockIdx.x * nlist;
     for (int base = 0; base < nlist; base += blockDim.x) {
         int c = base + threadIdx.x;
         if (c < nlist) {
-            unsigned long long key = make_key(row[c], (uint32_t)c);
+            unsigned long long key = SIGNED ? ((unsigned long long)ordered_bits(row[c]) << 32) | (uint32_t)c
+                                            : make_key(row[c], (uint32_t)c);
             if (key < tau) {
                 if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
             }
@@ -101,19 +111,33 @@ __global__ void __launch_bounds__(256) select_probes_kernel(const float* __restr
     topk_finalize<256>(t, nprobe);
     const int64_t q = q0 + blockIdx.x;
     for (int i = threadIdx.x; i < nprobe; i += blockDim.x) {
-        unsigned long long key = i < cnt ? buf[i] : kKeyPad;
+        unsigned long long key = i < cnt ? buf[i] : t.pad;
         probe_ids[q * nprobe + i] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
-        probe_d[q * nprobe + i] = __uint_as_float((uint32_t)(key >> 32));
+        probe_d[q * nprobe + i] = SIGNED ? from_ordered_bits((uint32_t)(key >> 32)) : __uint_as_float((uint32_t)(key >> 32));
     }
 }
 
 }  // namespace
 
+namespace {
+__global__ void negate_kernel(const float* __restrict__ in, float* __restrict__ out, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = -in[i];
+}
+}  // namespace
+
+// out[i] = -in[i]: the filtering stage of the inner-product path keeps -(q.c); callers see q.c.
+cudaError_t launch_negate(const float* in, float* out, int64_t n, cudaStream_t st) {
+    negate_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(in, out, n);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,
                           float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
                           int* status, cudaStream_t st, int64_t* launches) {
     // tensor-core proposal + exact decision when the shape allows it (16-byte aligned rows)
-    const bool mma = ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
+    const bool ip = ix->metric == IVFPQ_METRIC_IP;   // the tensor-core path and its error bound are written for L2
+    const bool mma = !ip && ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
                      (reinterpret_cast<uintptr_t>(ix->cent) & 15) == 0;
     for (int64_t q0 = 0; q0 < nq; q0 += qchunk) {
         const int nqc = (int)((nq - q0 < qchunk) ? (nq - q0) : qchunk);
@@ -123,8 +147,13 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
             if (e != cudaErrorNotSupported) return e;
         }
         dim3 grid((ix->nlist + TC - 1) / TC, (nqc + TQ - 1) / TQ);
-        coarse_dist_kernel<<<grid, 256, 0, st>>>(queries, q0, nqc, ix->cent, ix->nlist, ix->d, coarse_tile);
-        select_probes_kernel<<<nqc, 256, 0, st>>>(coarse_tile, ix->nlist, nprobe, probe_ids, probe_d, q0, status);
+        if (ip) {
+            coarse_dist_kernel<true><<<grid, 256, 0, st>>>(queries, q0, nqc, ix->cent, ix->nlist, ix->d, coarse_tile);
+            select_probes_kernel<true><<<nqc, 256, 0, st>>>(coarse_tile, ix->nlist, nprobe, probe_ids, probe_d, q0, status);
+        } else {
+            coarse_dist_kernel<false><<<grid, 256, 0, st>>>(queries, q0, nqc, ix->cent, ix->nlist, ix->d, coarse_tile);
+            select_probes_kernel<false><<<nqc, 256, 0, st>>>(coarse_tile, ix->nlist, nprobe, probe_ids, probe_d, q0, status);
+        }
         *launches += 2;
     }
     return cudaGetLastError();
@@ -169,6 +198,7 @@ extern "C" int ivfpq_probe_static(const ivfpq_index_t* index, const float* queri
     if (!index || !queries || !probe_ids || !probe_d) return IVFPQ_ERR_INVALID_ARGUMENT;
     if (nq <= 0 || nprobe <= 0) return IVFPQ_ERR_INVALID_ARGUMENT;
     if (nprobe > index->nlist || nprobe > IVFPQ_MAX_NPROBE || nq > (int64_t)1 << 24) return IVFPQ_ERR_UNSUPPORTED;
+    if (index->metric != IVFPQ_METRIC_L2) return IVFPQ_ERR_UNSUPPORTED;
     if (index->nlist > IVFPQ_STATIC_MAX_NLIST) return IVFPQ_ERR_STATIC_LIMIT;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return IVFPQ_ERR_CUDA;

@@ -25,6 +25,7 @@ inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a -
 // Host-side handle.  All pointers are device pointers into caller-owned memory.
 struct ivfpq_index {
     int32_t d, nlist, nsub, dsub, ksub;
+    int32_t metric;           // IVFPQ_METRIC_*
     int64_t ntotal;
     const float* cent;        // [nlist][d]
     const float* cb;          // [nsub][ksub][dsub]
@@ -119,6 +120,7 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
 cudaError_t launch_entry_stats(const ivfpq_index* ix, const uint8_t* codes, const float* queries, int64_t nq,
                                const int64_t* nbr, int k, int32_t* usage, unsigned long long* rank_hist, int* status,
                                cudaStream_t st);
+cudaError_t launch_negate(const float* in, float* out, int64_t n, cudaStream_t st);
 cudaError_t launch_thresholds(const float* queries, int64_t nq, int nsub, const ivfpq_threshold_model_t* m,
                               float* radius, cudaStream_t st);
 cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws, cudaStream_t st,

@@ -14,8 +14,10 @@ struct ScanParams {
     const int64_t* list_off;
     const int64_t* list_blk;
     int d, nlist, nsub, dsub, ksub, nw;
+    int vec16;   // generic layout: 1 = code words grouped by four (16-byte lane loads)
     const float* queries;
     const int32_t* probe_ids;
+    const float* probe_d;   // filtering value per probe; inner-product path: -(q.c), the start of every sum
     int nprobe;
     const float* radius;
     int radius_mode;

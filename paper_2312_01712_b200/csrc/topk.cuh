@@ -25,11 +25,23 @@ struct CtaGroup {
     __device__ __forceinline__ static void sync() { __syncthreads(); }
 };
 
+// Keys of values that may be negative (the inner-product path ranks by -similarity): an
+// order-preserving map of every fp32 to uint32 takes the place of the raw bits; -0 counts as +0.
+constexpr unsigned long long kKeyPadSigned = 0xFF800000FFFFFFFFull;  // ordered_bits(+inf), id -1
+__device__ __forceinline__ uint32_t ordered_bits(float v) {
+    const uint32_t u = __float_as_uint(__fadd_rn(v, 0.0f));
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t o) {
+    return __uint_as_float((o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o);
+}
+
 struct TopkState {
     unsigned long long* buf;  // [kTopkCap] shared memory
     int* cnt;                 // shared
     unsigned long long* tau;  // shared: a candidate is kept only if key < *tau
     int* hist;                // [kTopkHistInts] shared
+    unsigned long long pad = kKeyPad;  // the key that sorts after every real key (kKeyPadSigned for ordered_bits keys)
 };
 
 __device__ __forceinline__ unsigned long long make_key(float dist, uint32_t low) {
@@ -39,7 +51,7 @@ __device__ __forceinline__ unsigned long long make_key(float dist, uint32_t low)
 __device__ __forceinline__ void topk_init(const TopkState& t) {
     if (threadIdx.x == 0) {
         *t.cnt = 0;
-        *t.tau = kKeyPad;
+        *t.tau = t.pad;
     }
     __syncthreads();
 }

@@ -61,7 +61,7 @@ def test_derived_bytes_and_description_validation(L):
     # 2 + 0 + 2 blocks of 32 points x 1 word x 4 bytes, plus two list tables, 256-byte granules
     assert n >= 4 * 32 * 4 + 2 * 4 * 8 and n % 256 == 0
     assert L.ivfpq_index_derived_bytes(None) == 0
-    for bad in (dict(d=9), dict(ksub=257), dict(nsub=0), dict(metric=1), dict(ntotal=99),
+    for bad in (dict(d=9), dict(ksub=257), dict(nsub=0), dict(metric=2), dict(ntotal=99),
                 dict(offsets=[0, 50, 40, 100]), dict(offsets=[1, 40, 100]), dict(nsub=65, dsub=1, d=65),
                 dict(nsub=1, dsub=17, d=17)):
         assert L.ivfpq_index_derived_bytes(ctypes.byref(make_desc(**bad))) == 0, bad
