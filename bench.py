@@ -29,7 +29,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from ivfpq_inputs import CONFIGS, build_index_streamed, calibrate_radius, recall_1_at_k, recall_at_k  # noqa: E402
+import dataclasses  # noqa: E402
+
+from ivfpq_inputs import (CONFIGS, build_index_streamed, calibrate_radius, calibrate_radius_ip,  # noqa: E402
+                          recall_1_at_k, recall_at_k)
 from ivfpq_inputs import generators as G  # noqa: E402
 from ivfpq_inputs.groundtruth import ExactKnnAccumulator  # noqa: E402
 
@@ -131,16 +134,22 @@ def max_over_ranks(total_ms: float, dist, device) -> float:
     return float(t.item())
 
 
-def build_workload(name: str, device: str, nq: int | None, query_seed_offset: int = 0):
-    """Index + queries + exact neighbours + calibrated radii for one of the synthetic configs."""
+def build_workload(name: str, device: str, nq: int | None, query_seed_offset: int = 0, metric: int = 0):
+    """Index + queries + exact neighbours + calibrated radii for one of the synthetic configs.
+    metric 1: the same index (clusters and codebooks trained under L2) searched by inner product,
+    with exact maximum-inner-product neighbours as the ground truth."""
     cfg = rank_config(name, nq, query_seed_offset)
     t0 = time.time()
     spec = G.make_mixture(cfg, device)
     q = G.queries(cfg, spec)
-    acc = ExactKnnAccumulator(q, cfg.k)
+    acc = ExactKnnAccumulator(q, cfg.k, metric=metric)
     index = build_index_streamed(cfg, spec, on_chunk=acc.add)
     true_ids, _ = acc.result()
-    radius = calibrate_radius(index, G.calibration_queries(cfg, spec, 1000))
+    if metric == 1:
+        index = dataclasses.replace(index, metric=1)
+        radius = calibrate_radius_ip(index, G.calibration_queries(cfg, spec, 1000))
+    else:
+        radius = calibrate_radius(index, G.calibration_queries(cfg, spec, 1000))
     log(f"[bench] built {name}: N={index.ntotal} nlist={index.nlist} {index.nsub}x{index.dsub} "
         f"nq={q.shape[0]} in {time.time() - t0:.1f}s on {device}")
     return cfg, index, q.cpu().numpy(), true_ids, radius
@@ -183,6 +192,8 @@ SCORE_NAMES = {"distance": 0, "hit_count": 1, "reward_penalty": 2}
 
 def scan_kernel_name(index) -> str:
     """Name of the kernel the library picks for this index (same rule as ivfpq_index_load)."""
+    if getattr(index, "metric", 0) == 1:
+        return "scan_ip_kernel"
     if (index.nsub, index.dsub) == (16, 8):
         forced = os.environ.get("IVFPQ_SCAN_KERNEL")
         wide = forced == "warps32" or (forced != "warps16" and index.ntotal // index.nlist >= 2048)
@@ -219,7 +230,8 @@ def run_cuda(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     lib.load_library()
-    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq, query_seed_offset=rank)
+    metric = 1 if args.metric == "ip" else 0
+    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq, query_seed_offset=rank, metric=metric)
     nprobe = args.nprobe or cfg.nprobes[len(cfg.nprobes) // 2]
     k = cfg.k
     nq = q_np.shape[0]
@@ -327,10 +339,11 @@ def run_cuda(args):
         "config": {"workload": f"{cfg.name}: N={index.ntotal} D={index.d} nlist={index.nlist} "
                                f"PQ {index.nsub}x{index.dsub} (uint8 codes), nq={nq}/GPU, nprobe={nprobe}, k={k}, "
                                f"sparse search at radius scale {scale}"
-                               + ("" if score == 0 else f", ranked by {args.score}"),
+                               + ("" if score == 0 else f", ranked by {args.score}")
+                               + ("" if metric == 0 else ", inner-product similarity"),
                    "l2": "512 MiB buffer written between timed iterations (L2 flush)",
                    "parallelism": "replicas only (index replicated, queries split)" if world > 1 else "1 GPU",
-                   "radius_scale": scale, "nprobe": nprobe, "score": args.score},
+                   "radius_scale": scale, "nprobe": nprobe, "score": args.score, "similarity": args.metric},
         "recall@100": {"sparse": round(r_sparse, 4), "dense": round(r_dense, 4),
                        "R1@100_sparse": round(r1_sparse, 4), "R1@100_dense": round(r1_dense, 4)},
         "dense_queries_per_s": nq * world * dense_steps / (dense_ms * 1e-3),
@@ -345,7 +358,7 @@ def run_cuda(args):
                      "peak_source": f"of {peak_src}", "algorithmic_bytes_per_launch": int(scan_bytes),
                      "visits_per_launch": int(visits),
                      "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload)
-                     if (args.nq is None and args.nprobe == 0 and score == 0) else None},
+                     if (args.nq is None and args.nprobe == 0 and score == 0 and metric == 0) else None},
         "gather_roofline": {"bound": "shared-memory gathers", "achieved": gather_rate, "peak": gather_peak,
                             "unit": "Ggather/s", "frac": gather_rate / gather_peak,
                             "peak_source": f"{props.multi_processor_count} SMs x 32 lanes x {clk:.0f} MHz"},
@@ -385,7 +398,8 @@ def run_reference(args):
         return
     import oracle
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"      # input generation only
-    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq)
+    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq,
+                                                        metric=1 if args.metric == "ip" else 0)
     nprobe = args.nprobe or cfg.nprobes[len(cfg.nprobes) // 2]
     k = cfg.k
     sample = min(args.cpu_sample, q_np.shape[0])
@@ -425,6 +439,8 @@ def main():
     ap.add_argument("--nq", type=int, default=None)
     ap.add_argument("--cpu-sample", type=int, default=10000, help="queries timed on the CPU oracle")
     ap.add_argument("--ref-scale", type=float, default=1.0)
+    ap.add_argument("--metric", default="l2", choices=["l2", "ip"],
+                    help="similarity of the index (l2 = the headline path)")
     ap.add_argument("--score", default="distance", choices=sorted(SCORE_NAMES),
                     help="what the sparse search ranks by (distance = the headline path)")
     args = ap.parse_args()

@@ -18,6 +18,7 @@ from .index_build import (
     build_index,
     build_index_streamed,
     calibrate_radius,
+    calibrate_radius_ip,
     lossless_toy_index,
     load_index,
     save_index,
@@ -36,6 +37,7 @@ __all__ = [
     "build_index",
     "build_index_streamed",
     "calibrate_radius",
+    "calibrate_radius_ip",
     "lossless_toy_index",
     "load_index",
     "save_index",

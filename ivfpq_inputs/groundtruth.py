@@ -13,12 +13,14 @@ import torch
 
 
 class ExactKnnAccumulator:
-    """Running exact top-k (squared L2) of a fixed query set over base vectors
-    that arrive in chunks."""
+    """Running exact top-k (squared L2, or largest inner product with `metric=1`) of a fixed
+    query set over base vectors that arrive in chunks.  For the inner product the values kept
+    are the negated similarities, so that "smallest first" holds in both cases."""
 
-    def __init__(self, queries: torch.Tensor, k: int, block: int = 131072):
+    def __init__(self, queries: torch.Tensor, k: int, block: int = 131072, metric: int = 0):
         self.q = queries
         self.k = k
+        self.metric = metric
         self.block = block
         self.qn = (queries * queries).sum(1)
         nq = queries.shape[0]
@@ -29,7 +31,10 @@ class ExactKnnAccumulator:
         block = max(1024, min(self.block, (1 << 28) // max(1, self.q.shape[0])))
         for lo in range(0, x.shape[0], block):
             xb = x[lo:lo + block]
-            d = self.qn[:, None] - 2.0 * (self.q @ xb.T) + (xb * xb).sum(1)[None, :]
+            if self.metric == 1:
+                d = -(self.q @ xb.T)
+            else:
+                d = self.qn[:, None] - 2.0 * (self.q @ xb.T) + (xb * xb).sum(1)[None, :]
             kk = min(self.k, xb.shape[0])
             dv, di = torch.topk(d, kk, dim=1, largest=False)
             di = di + (first_id + lo)

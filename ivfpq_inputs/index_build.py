@@ -195,6 +195,23 @@ def calibrate_radius(index: IvfPqIndex, calib_queries: torch.Tensor, entry_rank:
     return out
 
 
+def calibrate_radius_ip(index: IvfPqIndex, calib_queries: torch.Tensor, entry_rank: int = 64) -> np.ndarray:
+    """Base radius per subspace for the inner-product metric, where entry e is selected when
+    |q_s - e|^2 - |e|^2 = |q_s|^2 - 2 q_s.e <= R^2: sqrt of the mean `entry_rank`-th smallest value
+    of that expression over calibration queries (0 where the mean is negative: the spheres of
+    radius |e| alone already select more than `entry_rank` entries).  Returns [nsub] fp32."""
+    dev = calib_queries.device
+    cb = torch.from_numpy(index.codebooks).to(dev)
+    rank = min(entry_rank, index.ksub)
+    out = np.empty(index.nsub, dtype=np.float32)
+    for s in range(index.nsub):
+        qs = calib_queries[:, s * index.dsub:(s + 1) * index.dsub]
+        v = (qs * qs).sum(1)[:, None] - 2.0 * (qs @ cb[s].T)
+        kth = torch.kthvalue(v, rank, dim=1).values
+        out[s] = float(torch.sqrt(torch.clamp(kth.mean(), min=0.0)))
+    return out
+
+
 def lossless_toy_index(seed: int, n: int, nlist: int, nsub: int, dsub: int, ksub: int = 256,
                        spread: float = 10.0):
     """A tiny index whose base vectors are *exactly* representable: every vector
