@@ -23,7 +23,11 @@ namespace ivfpq {
 
 namespace {
 
-constexpr int kLutGroupFloats = 256 * 32;  // one group table: 256 entries x 32 columns
+// Floats of one group table: 256 entries x 32 columns; a group of width 4 or less keeps one
+// compact copy (256 x w: its few look-ups may collide on a bank, but it costs 8 KB less per subspace).
+__host__ __device__ constexpr int row_stride(int w) { return w <= 4 ? w : 32; }
+__host__ __device__ constexpr int group_floats(int w) { return 256 * row_stride(w); }
+
 
 __host__ __device__ constexpr int lane_bytes(int w) { return w >= 16 ? w : (w == 8 ? 8 : (w > 0 ? 4 : 0)); }
 
@@ -35,14 +39,19 @@ struct Groups {
     __host__ __device__ static constexpr int width(int g) { return g == 0 ? W0 : (g == 1 ? W1 : W2); }
     __host__ __device__ static constexpr int s0(int g) { return g == 0 ? 0 : (g == 1 ? W0 : W0 + W1); }
     // byte offset of group g's chunk inside a 32-point block
+    // float offset of group g's table inside the table region, and the size of the region
+    __host__ __device__ static constexpr int lut_off(int g) {
+        return g == 0 ? 0 : (g == 1 ? group_floats(W0) : group_floats(W0) + group_floats(W1));
+    }
+    static constexpr int kLutFloats = group_floats(W0) + (W1 > 0 ? group_floats(W1) : 0) + (W2 > 0 ? group_floats(W2) : 0);
     __host__ __device__ static constexpr int chunk_off(int g) {
         return 32 * (g == 0 ? 0 : (g == 1 ? lane_bytes(W0) : lane_bytes(W0) + lane_bytes(W1)));
     }
 };
 
-__host__ __device__ inline size_t rot_smem_bytes(int ngroups, int d, int nprobe, bool dbg) {
+__host__ __device__ inline size_t rot_smem_bytes(int lut_floats, int d, int nprobe, bool dbg) {
     size_t b = (size_t)kTopkCap * 8;
-    b += (size_t)ngroups * kLutGroupFloats * 4;
+    b += (size_t)lut_floats * 4;
     b += align_up((size_t)d * 4, 16);
     b += IVFPQ_MAX_NSUB * 4;
     b += 32 + kTopkHistInts * 4;
@@ -57,7 +66,8 @@ __device__ __forceinline__ void build_group(float* __restrict__ lutg, const floa
                                             const float* __restrict__ res_g, const float* __restrict__ r2_g,
                                             int ksub, bool dense, int score, float P, uint32_t* hitmask_g) {
     constexpr int EP = NT / W;      // entries per pass
-    constexpr int NCOPY = 32 / W;
+    constexpr int RS = row_stride(W);
+    constexpr int NCOPY = RS / W;
     const int t = threadIdx.x;
     const int c = t & (W - 1);
     const int u = t / W;
@@ -100,7 +110,7 @@ __device__ __forceinline__ void build_group(float* __restrict__ lutg, const floa
             hit = dense || d2 <= thr;
         }
         const float val = table_value(score, hit, d2, thr, P);
-        float* row = lutg + e * 32 + c;
+        float* row = lutg + e * RS + c;
 #pragma unroll
         for (int it = 0; it < NCOPY; ++it) {
             const int copy = (it + usub) & (NCOPY - 1);  // lanes of a warp write different columns
@@ -119,7 +129,7 @@ __device__ __forceinline__ void gather_group(const float* __restrict__ lutg, con
 #pragma unroll
     for (int i = 0; i < W; ++i) {
         const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 0xFFu;
-        acc += lutg[code * 32 + (lane ^ i)];
+        acc += lutg[code * row_stride(W) + ((lane ^ i) & (row_stride(W) - 1))];
         if (DBG) {
             const int s = s0 + ((lane ^ i) & (W - 1));
             hs |= (unsigned long long)((hitmask[s * 8 + (code >> 5)] >> (code & 31)) & 1u) << s;
@@ -149,7 +159,7 @@ __device__ __forceinline__ void load_group_codes(const unsigned char* __restrict
 }
 
 template <int W0, int W1, int W2, int DSUB, int NT, bool DBG>
-__global__ void __launch_bounds__(NT) scan_rot_kernel(const ScanParams p) {
+__global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const ScanParams p) {
     using GR = Groups<W0, W1, W2>;
     constexpr int kWarps = NT / 32;
     constexpr int kBlocksPerWarpRound = 1024 / NT;       // 1024 candidates per round, CTA-wide
@@ -164,7 +174,7 @@ __global__ void __launch_bounds__(NT) scan_rot_kernel(const ScanParams p) {
 
     unsigned long long* kbuf = reinterpret_cast<unsigned long long*>(smem);
     float* lut = reinterpret_cast<float*>(smem + (size_t)kTopkCap * 8);
-    float* res = lut + (size_t)GR::kNum * kLutGroupFloats;
+    float* res = lut + (size_t)GR::kLutFloats;
     float* r2 = res + align_up((size_t)d * 4, 16) / 4;
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + IVFPQ_MAX_NSUB);
     int* cnt_p = reinterpret_cast<int*>(tau_p + 1);
@@ -220,11 +230,11 @@ __global__ void __launch_bounds__(NT) scan_rot_kernel(const ScanParams p) {
         // ---- selective tables, one per group ----
         build_group<W0, DSUB, NT, DBG>(lut, p.cbt, res, r2, ksub, p.dense, p.score, P, hitmask);
         if constexpr (W1 > 0)
-            build_group<W1, DSUB, NT, DBG>(lut + kLutGroupFloats, p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
+            build_group<W1, DSUB, NT, DBG>(lut + GR::lut_off(1), p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
                                            res + GR::s0(1) * DSUB, r2 + GR::s0(1), ksub, p.dense, p.score, P,
                                            hitmask + GR::s0(1) * 8);
         if constexpr (W2 > 0)
-            build_group<W2, DSUB, NT, DBG>(lut + 2 * kLutGroupFloats, p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
+            build_group<W2, DSUB, NT, DBG>(lut + GR::lut_off(2), p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
                                            res + GR::s0(2) * DSUB, r2 + GR::s0(2), ksub, p.dense, p.score, P,
                                            hitmask + GR::s0(2) * 8);
         __syncthreads();
@@ -258,9 +268,9 @@ __global__ void __launch_bounds__(NT) scan_rot_kernel(const ScanParams p) {
                 float acc = 0.0f;
                 unsigned long long hs = 0;
                 gather_group<W0, DBG>(lut, w0, lane, 0, hitmask, acc, hs);
-                if constexpr (W1 > 0) gather_group<W1, DBG>(lut + kLutGroupFloats, w1, lane, GR::s0(1), hitmask, acc, hs);
+                if constexpr (W1 > 0) gather_group<W1, DBG>(lut + GR::lut_off(1), w1, lane, GR::s0(1), hitmask, acc, hs);
                 if constexpr (W2 > 0)
-                    gather_group<W2, DBG>(lut + 2 * kLutGroupFloats, w2, lane, GR::s0(2), hitmask, acc, hs);
+                    gather_group<W2, DBG>(lut + GR::lut_off(2), w2, lane, GR::s0(2), hitmask, acc, hs);
                 const int64_t pos = blk * kPointsPerBlock + lane;
                 if (pos < len) {
                     if (DBG) {
@@ -299,7 +309,7 @@ __global__ void __launch_bounds__(NT) scan_rot_kernel(const ScanParams p) {
 
 template <int W0, int W1, int W2, int DSUB, int NT>
 cudaError_t launch_rot(const ScanParams& sp, int64_t grid, bool debug, int nprobe, cudaStream_t st) {
-    const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kNum, sp.d, nprobe, debug);
+    const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kLutFloats, sp.d, nprobe, debug);
     cudaError_t e;
     if (debug) {
         auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, true>;
@@ -340,8 +350,10 @@ bool rot_supported(int nsub, int dsub) {
 
 cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, bool debug, int nprobe,
                             cudaStream_t st) {
-    if (ix->nsub == 48 && ix->dsub == 2) return launch_rot<32, 16, 0, 2, 256>(sp, grid, debug, nprobe, st);
-    if (ix->nsub == 50 && ix->dsub == 4) return launch_rot<32, 16, 2, 4, 256>(sp, grid, debug, nprobe, st);
+    // The wide shapes run 512 threads per CTA at 64 registers, two CTAs per SM (32 warps): the table
+    // build waits on codebook loads from L2 and needs the warps to hide them.
+    if (ix->nsub == 48 && ix->dsub == 2) return launch_rot<32, 16, 0, 2, 512>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 50 && ix->dsub == 4) return launch_rot<32, 16, 2, 4, 512>(sp, grid, debug, nprobe, st);
     if (ix->nsub == 8 && ix->dsub == 4) return launch_rot<8, 0, 0, 4, 256>(sp, grid, debug, nprobe, st);
     if (ix->nsub == 12 && ix->dsub == 2) return launch_rot<8, 4, 0, 2, 256>(sp, grid, debug, nprobe, st);
     return cudaErrorNotSupported;
