@@ -31,8 +31,8 @@ if ROOT not in sys.path:
 
 import dataclasses  # noqa: E402
 
-from ivfpq_inputs import (CONFIGS, build_index_streamed, calibrate_radius, calibrate_radius_ip,  # noqa: E402
-                          recall_1_at_k, recall_at_k)
+from ivfpq_inputs import (CONFIGS, DensityAccumulator, build_index_streamed, calibrate_radius,  # noqa: E402
+                          calibrate_radius_ip, fit_threshold_model, recall_1_at_k, recall_at_k)
 from ivfpq_inputs import generators as G  # noqa: E402
 from ivfpq_inputs.groundtruth import ExactKnnAccumulator  # noqa: E402
 
@@ -134,7 +134,8 @@ def max_over_ranks(total_ms: float, dist, device) -> float:
     return float(t.item())
 
 
-def build_workload(name: str, device: str, nq: int | None, query_seed_offset: int = 0, metric: int = 0):
+def build_workload(name: str, device: str, nq: int | None, query_seed_offset: int = 0, metric: int = 0,
+                   dynamic: bool = False):
     """Index + queries + exact neighbours + calibrated radii for one of the synthetic configs.
     metric 1: the same index (clusters and codebooks trained under L2) searched by inner product,
     with exact maximum-inner-product neighbours as the ground truth."""
@@ -143,8 +144,28 @@ def build_workload(name: str, device: str, nq: int | None, query_seed_offset: in
     spec = G.make_mixture(cfg, device)
     q = G.queries(cfg, spec)
     acc = ExactKnnAccumulator(q, cfg.k, metric=metric)
-    index = build_index_streamed(cfg, spec, on_chunk=acc.add)
+    on_chunk, dens, acc_cal, cal_q = acc.add, None, None, None
+    if dynamic:
+        # density maps of the base projections and exact neighbours of the training queries, gathered
+        # in the same pass over the base vectors (unit-norm data: every projection lies in [-1, 1]^2)
+        if cfg.dsub != 2 or not cfg.normalize:
+            raise SystemExit("--dynamic-radius needs 2-d subspaces on unit-norm data (workload c3)")
+        lo = torch.full((cfg.nsub, 2), -1.0, device=device)
+        dens = DensityAccumulator(cfg.nsub, 100, (lo, -lo))
+        cal_q = G.calibration_queries(cfg, spec, 1000)
+        acc_cal = ExactKnnAccumulator(cal_q, cfg.k)
+
+        def on_chunk(first_id, x):
+            acc.add(first_id, x)
+            acc_cal.add(first_id, x)
+            dens.add(x)
+    index = build_index_streamed(cfg, spec, on_chunk=on_chunk)
     true_ids, _ = acc.result()
+    if dynamic:
+        d_map, origin, inv_cell = dens.result()
+        model = fit_threshold_model(index, d_map, origin, inv_cell, cal_q, acc_cal.result()[0], degree=2)
+        log(f"[bench] built {name} with a threshold model (100 x 100 maps, degree 2) in {time.time() - t0:.1f}s")
+        return cfg, index, q.cpu().numpy(), true_ids, model
     if metric == 1:
         index = dataclasses.replace(index, metric=1)
         radius = calibrate_radius_ip(index, G.calibration_queries(cfg, spec, 1000))
@@ -231,13 +252,24 @@ def run_cuda(args):
 
     lib.load_library()
     metric = 1 if args.metric == "ip" else 0
-    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq, query_seed_offset=rank, metric=metric)
+    dynamic = bool(args.dynamic_radius)
+    if dynamic and (metric != 0 or args.score != "distance"):
+        raise SystemExit("--dynamic-radius goes with the L2 distance search")
+    cfg, index, q_np, true_ids, radius = build_workload(args.workload, dev, args.nq, query_seed_offset=rank,
+                                                        metric=metric, dynamic=dynamic)
     nprobe = args.nprobe or cfg.nprobes[len(cfg.nprobes) // 2]
     k = cfg.k
     nq = q_np.shape[0]
     h = lib.ivfpq_index_load(index, dev)
     qd = torch.from_numpy(q_np).to(dev)
-    rad_d = torch.from_numpy(radius).to(dev)
+    model = mh = None
+    if dynamic:
+        # query-specific thresholds from the density maps and the regressor, computed on the device
+        model, radius = radius, None
+        mh = lib.ThresholdModelHandle(model, dev)
+        rad_d = lib.ivfpq_query_thresholds(h, qd, mh)
+    else:
+        rad_d = torch.from_numpy(radius).to(dev)
     out = (torch.empty((nq, k), dtype=torch.float32, device=dev), torch.empty((nq, k), dtype=torch.int32, device=dev))
 
     def dense_ids():
@@ -262,6 +294,8 @@ def run_cuda(args):
     lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_TIMING, 1)
 
     def step_sparse():
+        if dynamic:
+            lib.ivfpq_query_thresholds(h, qd, mh, out=rad_d)
         lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=scale, out=out, score=score)
 
     def step_dense():
@@ -294,7 +328,7 @@ def run_cuda(args):
     sampler = ClockSampler(local_rank)
     stages = []
     total_ms = timed(step_sparse, args.steps, args.warmup, sampler, stages)
-    launches = lib.ivfpq_last_launch_count(h) * args.steps
+    launches = (lib.ivfpq_last_launch_count(h) + (1 if dynamic else 0)) * args.steps
     dense_ms = timed(step_dense, max(3, args.steps // 4), 3)
     dense_steps = max(3, args.steps // 4)
 
@@ -303,13 +337,34 @@ def run_cuda(args):
     odh = torch.empty((nq, k), dtype=torch.float32).pin_memory()
     oih = torch.empty((nq, k), dtype=torch.int32).pin_memory()
 
+    qd2 = torch.empty_like(qd)
+
     def step_host():
-        lib.ivfpq_search_host(h, qh, nprobe, k, odh, oih, radius=rad_d, scale=scale, score=score)
+        if dynamic:   # the thresholds need the queries on the device before the search call
+            qd2.copy_(qh, non_blocking=True)
+            lib.ivfpq_query_thresholds(h, qd2, mh, out=rad_d)
+            lib.ivfpq_search_sparse(h, qd2, nprobe, rad_d, k, scale=scale, out=out)
+            odh.copy_(out[0], non_blocking=True)
+            oih.copy_(out[1], non_blocking=True)
+        else:
+            lib.ivfpq_search_host(h, qh, nprobe, k, odh, oih, radius=rad_d, scale=scale, score=score)
 
     lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_TIMING, 0)
     e2e_steps = max(3, args.steps // 4)
     e2e_ms = timed(step_host, e2e_steps, 3)
     assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
+
+    # the paper's comparison (Sec. 6.3 "Effectiveness of Dynamic Threshold Strategy"): one static
+    # threshold per subspace set to the smallest / largest of the query-specific ones
+    dyn_report = None
+    if dynamic:
+        lib.ivfpq_query_thresholds(h, qd, mh, out=rad_d)
+        scaled = rad_d * scale
+        dyn_report = {"threshold_min_mean_max": [float(scaled.min()), float(scaled.mean()), float(scaled.max())]}
+        for name, stat in (("static_small", scaled.min(dim=0).values.contiguous()), ("static_large", scaled.max(dim=0).values.contiguous())):
+            ids = lib.ivfpq_search_sparse(h, qd, nprobe, stat, k)[1].cpu().numpy()
+            ms = timed(lambda: lib.ivfpq_search_sparse(h, qd, nprobe, stat, k, out=out), 5, 3)
+            dyn_report[name] = {"recall@100": round(recall_at_k(ids, true_ids), 4), "queries_per_s": nq * world * 5 / (ms * 1e-3)}
 
     if rank != 0:
         if dist is not None:
@@ -330,7 +385,7 @@ def run_cuda(args):
     gather_peak = props.multi_processor_count * 32 * clk * 1e6 / 1e9            # G gathers/s
     gather_rate = scan_bytes / (scan_ms * 1e-3) / 1e9                            # one gather per code byte
 
-    cpu = cpu_baseline(index, q_np, nprobe, k, radius, scale, args.cpu_sample, score)
+    cpu = cpu_baseline(index, q_np, nprobe, k, radius, scale, args.cpu_sample, score, model)
 
     line = {
         "metric": METRIC, "value": nq * world * args.steps / (total_ms * 1e-3), "unit": UNIT,
@@ -340,7 +395,8 @@ def run_cuda(args):
                                f"PQ {index.nsub}x{index.dsub} (uint8 codes), nq={nq}/GPU, nprobe={nprobe}, k={k}, "
                                f"sparse search at radius scale {scale}"
                                + ("" if score == 0 else f", ranked by {args.score}")
-                               + ("" if metric == 0 else ", inner-product similarity"),
+                               + ("" if metric == 0 else ", inner-product similarity")
+                               + ("" if not dynamic else ", query-specific thresholds (density map + regressor) computed in the step"),
                    "l2": "512 MiB buffer written between timed iterations (L2 flush)",
                    "parallelism": "replicas only (index replicated, queries split)" if world > 1 else "1 GPU",
                    "radius_scale": scale, "nprobe": nprobe, "score": args.score, "similarity": args.metric},
@@ -364,6 +420,8 @@ def run_cuda(args):
                             "peak_source": f"{props.multi_processor_count} SMs x 32 lanes x {clk:.0f} MHz"},
         "cpu_baseline": cpu,
     }
+    if dyn_report is not None:
+        line["dynamic_threshold"] = dyn_report
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -381,11 +439,15 @@ class _Null:
 # the CPU oracle: cpu_baseline leg and --impl reference
 # --------------------------------------------------------------------------------------------
 
-def cpu_baseline(index, q_np, nprobe, k, radius, scale, sample, score=0):
+def cpu_baseline(index, q_np, nprobe, k, radius, scale, sample, score=0, model=None):
     import oracle
     sample = min(sample, q_np.shape[0])
+    if model is not None:
+        radius = oracle.thresholds(index.d, index.nsub, index.dsub, q_np[:8], model)
     oracle.search(index, q_np[:8], nprobe, k, radius=radius, scale=scale, score=score)    # page in
     t0 = time.perf_counter()
+    if model is not None:
+        radius = oracle.thresholds(index.d, index.nsub, index.dsub, q_np[:sample], model)
     oracle.search(index, q_np[:sample], nprobe, k, radius=radius, scale=scale, score=score)
     dt = time.perf_counter() - t0
     return {"value": sample / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
@@ -439,6 +501,8 @@ def main():
     ap.add_argument("--nq", type=int, default=None)
     ap.add_argument("--cpu-sample", type=int, default=10000, help="queries timed on the CPU oracle")
     ap.add_argument("--ref-scale", type=float, default=1.0)
+    ap.add_argument("--dynamic-radius", action="store_true",
+                    help="query-specific thresholds from density maps + polynomial regressor (workload c3)")
     ap.add_argument("--metric", default="l2", choices=["l2", "ip"],
                     help="similarity of the index (l2 = the headline path)")
     ap.add_argument("--score", default="distance", choices=sorted(SCORE_NAMES),

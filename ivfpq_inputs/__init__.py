@@ -24,7 +24,8 @@ from .index_build import (
     save_index,
 )
 from .groundtruth import exact_knn, recall_at_k, recall_1_at_k
-from .thresholds import ThresholdModel, containing_thresholds, density_maps, fit_threshold_model
+from .thresholds import (DensityAccumulator, ThresholdModel, containing_thresholds, density_maps,
+                         fit_threshold_model)
 
 __all__ = [
     "CONFIGS",
@@ -46,6 +47,7 @@ __all__ = [
     "recall_1_at_k",
     "ThresholdModel",
     "containing_thresholds",
+    "DensityAccumulator",
     "density_maps",
     "fit_threshold_model",
 ]

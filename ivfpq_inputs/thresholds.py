@@ -35,25 +35,40 @@ def cell_index(x: torch.Tensor, origin: torch.Tensor, inv_cell: torch.Tensor, gr
     return torch.nan_to_num(t, nan=0.0).clamp_(0, grid - 1).to(torch.int64)
 
 
+class DensityAccumulator:
+    """Density maps of base vectors that arrive in chunks: `add(x)` per chunk [n, 2 * nsub],
+    `result()` = (density [nsub, grid, grid], origin [nsub, 2], inv_cell [nsub, 2]) as fp32 numpy.
+    extent: (lo [nsub, 2], hi [nsub, 2]) tensors on the device the counting runs on."""
+
+    def __init__(self, nsub: int, grid: int, extent: Tuple[torch.Tensor, torch.Tensor]):
+        self.lo, hi = extent
+        self.nsub, self.grid = nsub, grid
+        cell = (hi - self.lo) / grid
+        self.cell = torch.where(cell > 0, cell, torch.ones_like(cell))
+        self.inv = (1.0 / self.cell).to(torch.float32)
+        self.counts = torch.zeros((nsub, grid * grid), dtype=torch.float64, device=self.lo.device)
+
+    def add(self, x: torch.Tensor) -> None:
+        x = x.to(self.lo.device)
+        for s in range(self.nsub):
+            idx = cell_index(x[:, 2 * s:2 * s + 2], self.lo[s], self.inv[s], self.grid)
+            flat = idx[:, 1] * self.grid + idx[:, 0]
+            self.counts[s] += torch.bincount(flat, minlength=self.grid * self.grid).to(torch.float64)
+
+    def result(self):
+        area = (self.cell[:, 0] * self.cell[:, 1]).to(torch.float64)
+        dens = (self.counts / area[:, None]).reshape(self.nsub, self.grid, self.grid).to(torch.float32)
+        return dens.cpu().numpy(), self.lo.to(torch.float32).cpu().numpy(), self.inv.cpu().numpy()
+
+
 def density_maps(chunks: Iterable[torch.Tensor], nsub: int, grid: int,
                  extent: Tuple[torch.Tensor, torch.Tensor]):
     """chunks: base vectors [n, 2 * nsub] (any device); extent: (lo [nsub, 2], hi [nsub, 2]).
     Returns (density [nsub, grid, grid], origin [nsub, 2], inv_cell [nsub, 2]) as fp32 numpy."""
-    lo, hi = extent
-    dev = lo.device
-    cell = (hi - lo) / grid
-    cell = torch.where(cell > 0, cell, torch.ones_like(cell))
-    inv = (1.0 / cell).to(torch.float32)
-    counts = torch.zeros((nsub, grid * grid), dtype=torch.float64, device=dev)
+    acc = DensityAccumulator(nsub, grid, extent)
     for x in chunks:
-        x = x.to(dev)
-        for s in range(nsub):
-            idx = cell_index(x[:, 2 * s:2 * s + 2], lo[s], inv[s], grid)
-            flat = idx[:, 1] * grid + idx[:, 0]
-            counts[s] += torch.bincount(flat, minlength=grid * grid).to(torch.float64)
-    area = (cell[:, 0] * cell[:, 1]).to(torch.float64)
-    dens = (counts / area[:, None]).reshape(nsub, grid, grid).to(torch.float32)
-    return dens.cpu().numpy(), lo.to(torch.float32).cpu().numpy(), inv.cpu().numpy()
+        acc.add(x)
+    return acc.result()
 
 
 def containing_thresholds(index, queries: torch.Tensor, neighbour_ids: np.ndarray) -> np.ndarray:
