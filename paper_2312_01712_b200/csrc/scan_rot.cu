@@ -31,9 +31,16 @@ __host__ __device__ constexpr int group_floats(int w) { return 256 * row_stride(
 
 __host__ __device__ constexpr int lane_bytes(int w) { return w >= 16 ? w : (w == 8 ? 8 : (w > 0 ? 4 : 0)); }
 
+// Paired layout (shapes whose first two groups are 32 and 16 wide): the two tables share rows of
+// 256 bytes, [32 columns of group 0 | 32 columns of group 1], at a fixed address of the CTA's
+// shared window, so that a look-up address is {code, column offset} put together by one byte
+// permute and the base is an immediate of the load.
+constexpr uint32_t kPairWin = 0x5000;          // shared-window address of the paired tables (64 KB)
+constexpr int kPairRowFloats = 64;
+
 template <int W0, int W1, int W2>
 struct Groups {
-    static constexpr int kNum = (W0 > 0) + (W1 > 0) + (W2 > 0);
+    static constexpr bool kPaired = (W0 == 32 && W1 == 16);
     static constexpr int kNsub = W0 + W1 + W2;
     static constexpr int kBlockBytes = 32 * (lane_bytes(W0) + lane_bytes(W1) + lane_bytes(W2));
     __host__ __device__ static constexpr int width(int g) { return g == 0 ? W0 : (g == 1 ? W1 : W2); }
@@ -41,7 +48,12 @@ struct Groups {
     // byte offset of group g's chunk inside a 32-point block
     // float offset of group g's table inside the table region, and the size of the region
     __host__ __device__ static constexpr int lut_off(int g) {
+        if (kPaired) return g == 0 ? 0 : (g == 1 ? 32 : 256 * kPairRowFloats);
         return g == 0 ? 0 : (g == 1 ? group_floats(W0) : group_floats(W0) + group_floats(W1));
+    }
+    // floats between two rows of group g's table
+    __host__ __device__ static constexpr int stride(int g) {
+        return (kPaired && g < 2) ? kPairRowFloats : row_stride(width(g));
     }
     static constexpr int kLutFloats = group_floats(W0) + (W1 > 0 ? group_floats(W1) : 0) + (W2 > 0 ? group_floats(W2) : 0);
     __host__ __device__ static constexpr int chunk_off(int g) {
@@ -49,25 +61,28 @@ struct Groups {
     }
 };
 
-__host__ __device__ inline size_t rot_smem_bytes(int lut_floats, int d, int nprobe, bool dbg) {
-    size_t b = (size_t)kTopkCap * 8;
+// Bytes in front of the tables: candidate keys, residual, thresholds, counters, histogram.
+__host__ __device__ inline size_t rot_aux_bytes(int d) {
+    return (size_t)kTopkCap * 8 + align_up((size_t)d * 4, 16) + IVFPQ_MAX_NSUB * 4 + 32 + kTopkHistInts * 4;
+}
+
+// Dynamic shared memory of a launch.  Paired layout: everything up to the fixed table address
+// (whatever the window offset of the allocation turns out to be), the tables, the debug area.
+__host__ __device__ inline size_t rot_smem_bytes(bool paired, int lut_floats, int d, int nprobe, bool dbg) {
+    size_t b = paired ? (size_t)kPairWin : rot_aux_bytes(d);
     b += (size_t)lut_floats * 4;
-    b += align_up((size_t)d * 4, 16);
-    b += IVFPQ_MAX_NSUB * 4;
-    b += 32 + kTopkHistInts * 4;
     if (dbg) b += IVFPQ_MAX_NSUB * 8 * 4 + (size_t)(nprobe + 1) * 8;
     return b;
 }
 
 // Table of one group for one (query, cluster): thread t owns column c = t & (W-1) and the
 // entries u, u + NT/W, ... with u = t / W.
-template <int W, int DSUB, int NT, bool DBG>
+template <int W, int DSUB, int NT, bool DBG, int RS = row_stride(W)>
 __device__ __forceinline__ void build_group(float* __restrict__ lutg, const float* __restrict__ cbt_g,
                                             const float* __restrict__ res_g, const float* __restrict__ r2_g,
                                             int ksub, bool dense, int score, float P, uint32_t* hitmask_g) {
     constexpr int EP = NT / W;      // entries per pass
-    constexpr int RS = row_stride(W);
-    constexpr int NCOPY = RS / W;
+    constexpr int NCOPY = (RS == kPairRowFloats ? 32 : RS) / W;   // copies within the group's 32 (or w) columns
     const int t = threadIdx.x;
     const int c = t & (W - 1);
     const int u = t / W;
@@ -137,6 +152,43 @@ __device__ __forceinline__ void gather_group(const float* __restrict__ lutg, con
     }
 }
 
+// One look-up of the paired tables.  `word` holds four code bytes, `pack` the lane's column offsets
+// (lane ^ i) * 4 of the same four steps; T = the byte of both that belongs to this step, G = group.
+// The permute builds {0, 0, code, column offset} (the zero bytes are the replicated sign of the
+// column offset, which is below 128); the table address is the immediate.
+template <int T, int G>
+__device__ __forceinline__ float pair_gather(uint32_t word, uint32_t pack) {
+    uint32_t addr;
+    float v;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(addr) : "r"(word), "r"(pack), "n"(((12 + T) << 12) | ((12 + T) << 8) | (T << 4) | (4 + T)));
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"((int)kPairWin + G * 128) : "memory");
+    return v;
+}
+
+// Table values of NW code words (4 NW subspaces of group G) added to two running sums.
+template <int NW, int G>
+__device__ __forceinline__ void pair_gather_words(const uint32_t* words, const uint32_t* pk, float& a0, float& a1) {
+#pragma unroll
+    for (int j = 0; j < NW; ++j) {
+        a0 += pair_gather<0, G>(words[j], pk[j]);
+        a1 += pair_gather<1, G>(words[j], pk[j]);
+        a0 += pair_gather<2, G>(words[j], pk[j]);
+        a1 += pair_gather<3, G>(words[j], pk[j]);
+    }
+}
+
+// Stage dumps: the subspaces of a group in which the lane's point hit a selected entry.
+template <int W>
+__device__ __forceinline__ void hits_group(const uint32_t* words, int lane, int s0, const uint32_t* hitmask,
+                                           unsigned long long& hs) {
+#pragma unroll
+    for (int i = 0; i < W; ++i) {
+        const uint32_t code = (words[i >> 2] >> (8 * (i & 3))) & 0xFFu;
+        const int s = s0 + ((lane ^ i) & (W - 1));
+        hs |= (unsigned long long)((hitmask[s * 8 + (code >> 5)] >> (code & 31)) & 1u) << s;
+    }
+}
+
 template <int W>
 __device__ __forceinline__ void load_group_codes(const unsigned char* __restrict__ chunk, int lane,
                                                  uint32_t* words) {
@@ -172,15 +224,37 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
     const int lane = tid & 31;
     const int warp = tid >> 5;
 
+    // candidate keys | residual | thresholds | counters | histogram | tables | debug area; in the
+    // paired layout the tables start at the fixed window address kPairWin
     unsigned long long* kbuf = reinterpret_cast<unsigned long long*>(smem);
-    float* lut = reinterpret_cast<float*>(smem + (size_t)kTopkCap * 8);
-    float* res = lut + (size_t)GR::kLutFloats;
+    float* res = reinterpret_cast<float*>(smem + (size_t)kTopkCap * 8);
     float* r2 = res + align_up((size_t)d * 4, 16) / 4;
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + IVFPQ_MAX_NSUB);
     int* cnt_p = reinterpret_cast<int*>(tau_p + 1);
     int* hist_p = reinterpret_cast<int*>(tau_p + 4);
-    uint32_t* hitmask = reinterpret_cast<uint32_t*>(hist_p + kTopkHistInts);           // DBG only
+    size_t lut_at = rot_aux_bytes(d);
+    if constexpr (GR::kPaired) {
+        const uint32_t win = (uint32_t)__cvta_generic_to_shared(smem);
+        if (win + lut_at > kPairWin) {   // uniform: the layout does not fit this window offset
+            if (tid == 0) atomicOr(p.status, kFlagLayout);
+            return;
+        }
+        lut_at = kPairWin - win;
+    }
+    float* lut = reinterpret_cast<float*>(smem + lut_at);
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(lut + GR::kLutFloats);             // DBG only
     long long* vprefix = reinterpret_cast<long long*>(hitmask + IVFPQ_MAX_NSUB * 8);   // DBG only
+    // paired layout: column offsets (lane ^ i) * 4 of the 32 steps, four per register
+    uint32_t pk[GR::kPaired ? 8 : 1];
+    if constexpr (GR::kPaired) {
+#pragma unroll
+        for (int k4 = 0; k4 < 8; ++k4) {
+            uint32_t v = 0;
+#pragma unroll
+            for (int tt = 0; tt < 4; ++tt) v |= (uint32_t)(((lane ^ (4 * k4 + tt)) * 4) & 0xFF) << (8 * tt);
+            pk[k4] = v;
+        }
+    }
 
     const int64_t q = blockIdx.x / p.nsplit;
     const int split = blockIdx.x % p.nsplit;
@@ -228,9 +302,9 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
         __syncthreads();
 
         // ---- selective tables, one per group ----
-        build_group<W0, DSUB, NT, DBG>(lut, p.cbt, res, r2, ksub, p.dense, p.score, P, hitmask);
+        build_group<W0, DSUB, NT, DBG, GR::stride(0)>(lut, p.cbt, res, r2, ksub, p.dense, p.score, P, hitmask);
         if constexpr (W1 > 0)
-            build_group<W1, DSUB, NT, DBG>(lut + GR::lut_off(1), p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
+            build_group<W1, DSUB, NT, DBG, GR::stride(1)>(lut + GR::lut_off(1), p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
                                            res + GR::s0(1) * DSUB, r2 + GR::s0(1), ksub, p.dense, p.score, P,
                                            hitmask + GR::s0(1) * 8);
         if constexpr (W2 > 0)
@@ -267,8 +341,19 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
                 if constexpr (W2 > 0) load_group_codes<W2>(bp + GR::chunk_off(2), lane, w2);
                 float acc = 0.0f;
                 unsigned long long hs = 0;
-                gather_group<W0, DBG>(lut, w0, lane, 0, hitmask, acc, hs);
-                if constexpr (W1 > 0) gather_group<W1, DBG>(lut + GR::lut_off(1), w1, lane, GR::s0(1), hitmask, acc, hs);
+                if constexpr (GR::kPaired) {
+                    float a0 = 0.0f, a1 = 0.0f;
+                    pair_gather_words<W0 / 4, 0>(w0, pk, a0, a1);
+                    pair_gather_words<W1 / 4, 1>(w1, pk, a0, a1);
+                    acc = a0 + a1;
+                    if (DBG) {
+                        hits_group<W0>(w0, lane, 0, hitmask, hs);
+                        hits_group<W1>(w1, lane, GR::s0(1), hitmask, hs);
+                    }
+                } else {
+                    gather_group<W0, DBG>(lut, w0, lane, 0, hitmask, acc, hs);
+                    if constexpr (W1 > 0) gather_group<W1, DBG>(lut + GR::lut_off(1), w1, lane, GR::s0(1), hitmask, acc, hs);
+                }
                 if constexpr (W2 > 0)
                     gather_group<W2, DBG>(lut + GR::lut_off(2), w2, lane, GR::s0(2), hitmask, acc, hs);
                 const int64_t pos = blk * kPointsPerBlock + lane;
@@ -309,7 +394,7 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
 
 template <int W0, int W1, int W2, int DSUB, int NT>
 cudaError_t launch_rot(const ScanParams& sp, int64_t grid, bool debug, int nprobe, cudaStream_t st) {
-    const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kLutFloats, sp.d, nprobe, debug);
+    const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kPaired, Groups<W0, W1, W2>::kLutFloats, sp.d, nprobe, debug);
     cudaError_t e;
     if (debug) {
         auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, true>;
