@@ -314,8 +314,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                     auto scan_blocks = [&](auto table_tag) {
                         constexpr int TABLE = decltype(table_tag)::value;
                         // one block: 16 look-ups per lane, stage dumps, candidate test
-                        auto one = [&](const uint4 cur, const int bpos) {
-                            const float acc = gather16<TABLE>(cur, pk);
+                        auto consider = [&](const uint4 cur, const float acc, const int bpos) {
                             if (bpos < m.len) {
                                 if (DBG) {
                                     unsigned long long hs = 0;
@@ -351,10 +350,30 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                         // round in which one of its candidates landed beyond the soft limit, which
                         // bounds the overshoot by 64 candidates per warp.
                         while (rem >= 2 && !halt) {
-                            one(n0, pos);
-                            if (rem > 2) n0 = __ldg(ptr + 2 * kStep);
-                            one(n1, pos + kWarps * kPointsPerBlock);
-                            if (rem > 3) n1 = __ldg(ptr + 3 * kStep);
+                            if constexpr (kNT == 512) {
+                                // L2-resident lists, four warps per scheduler: the look-ups of both blocks
+                                // first (32 independent loads, four running sums), then the two tests
+                                const float acc0 = gather16<TABLE>(n0, pk);
+                                const float acc1 = gather16<TABLE>(n1, pk);
+                                if (DBG) {   // the stage dumps read the codes: keep them until then
+                                    consider(n0, acc0, pos);
+                                    consider(n1, acc1, pos + kWarps * kPointsPerBlock);
+                                }
+                                const uint4 z = make_uint4(0, 0, 0, 0);
+                                if (rem > 2) n0 = __ldg(ptr + 2 * kStep);
+                                if (rem > 3) n1 = __ldg(ptr + 3 * kStep);
+                                if (!DBG) {
+                                    consider(z, acc0, pos);
+                                    consider(z, acc1, pos + kWarps * kPointsPerBlock);
+                                }
+                            } else {
+                                // lists streamed from HBM: each code register is refilled as soon as its
+                                // block has been consumed
+                                consider(n0, gather16<TABLE>(n0, pk), pos);
+                                if (rem > 2) n0 = __ldg(ptr + 2 * kStep);
+                                consider(n1, gather16<TABLE>(n1, pk), pos + kWarps * kPointsPerBlock);
+                                if (rem > 3) n1 = __ldg(ptr + 3 * kStep);
+                            }
                             if (kPf > 0) {
                                 if (rem > kPf + 1) prefetch_l2(ptr + (kPf + 1) * kStep);
                                 if (rem > kPf + 2) prefetch_l2(ptr + (kPf + 2) * kStep);
@@ -365,7 +384,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                             halt = __any_sync(0xFFFFFFFFu, stop);
                         }
                         if (rem == 1 && !halt) {
-                            one(n0, pos);
+                            consider(n0, gather16<TABLE>(n0, pk), pos);
                             rem = 0;
                             halt = __any_sync(0xFFFFFFFFu, stop);
                         }
