@@ -102,7 +102,7 @@ __device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[
     return a0 + a1;
 }
 
-template <int NT, bool DBG>
+template <int NT, bool DBG, bool SCORED>
 __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, const int64_t nitems) {
     constexpr int kNT = NT;
     constexpr int kWarps = Shape<NT>::kWarps;
@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
             }
             const int e = u + kEP * m;
             const bool hit = e < ksub && (p.dense || d2 <= thr);
-            const float val = table_value(p.score, hit, d2, thr, P);
+            const float val = table_value<SCORED>(p.score, hit, d2, thr, P);
             unsigned char* row = lutb + m * (kEP * kRowBytes);
             *reinterpret_cast<float*>(row + st_a) = val;
             *reinterpret_cast<float*>(row + st_b) = val;
@@ -405,23 +405,23 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
     }
 }
 
-template <int NT>
-cudaError_t launch_nt(const ScanParams& sp, int64_t grid, int64_t nitems, bool debug, cudaStream_t st) {
+template <int NT, bool DBG, bool SCORED>
+cudaError_t launch_inst(const ScanParams& sp, int64_t grid, int64_t nitems, cudaStream_t st) {
     // covers the table region (and the shared codebook of the 32-warp kernel) for any window offset
     const size_t smem = NT == 1024 ? (size_t)kCbWin + 65536 : (size_t)kCbWin;
-    cudaError_t e;
-    if (debug) {
-        auto kern = scan16x8_kernel<NT, true>;
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        kern<<<(unsigned)grid, NT, smem, st>>>(sp, nitems);
-    } else {
-        auto kern = scan16x8_kernel<NT, false>;
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        kern<<<(unsigned)grid, NT, smem, st>>>(sp, nitems);
-    }
+    auto kern = scan16x8_kernel<NT, DBG, SCORED>;
+    const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<(unsigned)grid, NT, smem, st>>>(sp, nitems);
     return cudaGetLastError();
+}
+
+// Instances: stage dumps (any score), count scores, distances only (the benchmarked path).
+template <int NT>
+cudaError_t launch_nt(const ScanParams& sp, int64_t grid, int64_t nitems, bool debug, cudaStream_t st) {
+    if (debug) return launch_inst<NT, true, true>(sp, grid, nitems, st);
+    if (sp.score != IVFPQ_SCORE_DISTANCE) return launch_inst<NT, false, true>(sp, grid, nitems, st);
+    return launch_inst<NT, false, false>(sp, grid, nitems, st);
 }
 
 }  // namespace
