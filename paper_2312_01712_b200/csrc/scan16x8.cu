@@ -61,9 +61,9 @@ static_assert(kSoftLimit + 2 * 1024 <= kCap && IVFPQ_MAX_K < kSoftLimit, "candid
 __host__ __device__ inline int scan16x8_aux_bytes(int nprobe, bool dbg) {
     int b = kCap * 8;                         // candidate keys
     b += kMetaCap * (int)sizeof(ProbeMeta);
-    b += kD * 4 + 2 * kD * 4 + 64;            // query, two centroids, squared thresholds
+    b += kD * 4 + 4 * kD * 4 + 64;            // query, four centroids, squared thresholds
     b += 32 + kQuickWords * 4;                // threshold, counters, compaction histogram
-    if (dbg) b += 2 * kW * 8 * 4 + (nprobe + 1) * 8;
+    if (dbg) b += 4 * kW * 8 * 4 + (nprobe + 1) * 8;
     return (b + 255) & ~255;
 }
 
@@ -76,7 +76,7 @@ __device__ __forceinline__ float lut_gather(uint32_t word, uint32_t pack) {
     uint32_t addr;
     float v;
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(addr) : "r"(word), "r"(pack), "n"(((12 + T) << 12) | ((12 + T) << 8) | (T << 4) | (4 + T)));
-    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"((int)kLutWin + TABLE * 128) : "memory");
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"((int)kLutWin + (TABLE >> 1) * 0x10000 + (TABLE & 1) * 128) : "memory");
     return v;
 }
 
@@ -133,17 +133,17 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
     ProbeMeta* meta = reinterpret_cast<ProbeMeta*>(a);
     a += kMetaCap * sizeof(ProbeMeta);
     float* qs = reinterpret_cast<float*>(a);
-    float* cent_s = qs + kD;          // [2][128]
-    float* r2 = cent_s + 2 * kD;      // [16]
-    a += kD * 4 + 2 * kD * 4 + 64;
+    float* cent_s = qs + kD;          // [4][128]
+    float* r2 = cent_s + 4 * kD;      // [16]
+    a += kD * 4 + 4 * kD * 4 + 64;
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(a);
     int* cnt_p = reinterpret_cast<int*>(a + 8);
     int* ntrans_p = cnt_p + 1;
     a += 32;
     int* hist_p = reinterpret_cast<int*>(a);
     a += kQuickWords * 4;
-    uint32_t* hitmask = reinterpret_cast<uint32_t*>(a);                        // DBG only: [2][16][8]
-    long long* vprefix = reinterpret_cast<long long*>(a + 2 * kW * 8 * 4);     // DBG only
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(a);                        // DBG only: [4][16][8]
+    long long* vprefix = reinterpret_cast<long long*>(a + 4 * kW * 8 * 4);     // DBG only
     TopkState t{kbuf, cnt_p, tau_p, hist_p};
 
     // ---- codebook: the first kRegEntries entries of a thread in registers, the others (32 warps
@@ -247,62 +247,110 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
             // ---- stage the metadata of the tile's clusters (the previous tile ended with a barrier) ----
             if (tid >= 128 && tid < 128 + nt) meta[tid - 128] = load_probe_meta(p, q, split + (t0 + tid - 128) * p.nsplit);
             if (DBG)
-                for (int i = tid; i < 2 * kW * 8; i += kNT) hitmask[i] = 0;
+                for (int i = tid; i < 4 * kW * 8; i += kNT) hitmask[i] = 0;
             __syncthreads();
             if (t0 == 0) {
                 P = miss_constant(p, r2);
                 thr = r2[c];
             }
 
-            // ---- prologue: centroids of the tile's first two clusters, table of the first ----
-            if (tid < 32) fetch_cent(meta[0].cl, cent_s, tid);
-            else if (tid < 64 && nt > 1) fetch_cent(meta[1].cl, cent_s + kD, tid - 32);
+            // The clusters are taken two at a time, their lists as one sequence of blocks dealt
+            // round-robin to the warps: the warps' block counts differ by one per pair of lists, not
+            // per list (the barrier that ends a phase waits for the slowest warp).
+            //   16 warps (kAhead): four tables (two 64 KB regions).  In one phase a warp builds its share
+            //   of the NEXT pair's tables and then scans its blocks of this pair: one barrier per pair,
+            //   and warps that build overlap with warps that scan.
+            //   32 warps: two tables.  Phase A builds the pair's tables, phase B scans its lists.
+            // Cluster j of the tile uses centroid slot and hit-mask buffer j & 3 (kAhead) or j & 1.
+            constexpr bool kAhead = kNT == 512;
+            constexpr int kSlots = kAhead ? 4 : 2;
+            auto table_of = [&](int jj) {   // table of cluster jj as a generic pointer
+                return lut_gen + (kAhead ? ((jj >> 1) & 1) * 0x10000 : 0) + (jj & 1) * 128;
+            };
+            auto build_cluster = [&](int jj) {
+                build(table_of(jj), cent_s + (jj & (kSlots - 1)) * kD, thr, P, hitmask + (jj & (kSlots - 1)) * kW * 8);
+            };
+            // ---- prologue: centroids of the tile's first clusters (and, kAhead, the first pair's tables) ----
+            if (tid < 32 * kSlots && (tid >> 5) < nt) fetch_cent(meta[tid >> 5].cl, cent_s + (tid >> 5) * kD, lane);
             cp_async_wait_all();
             __syncthreads();
-            build(lut_gen, cent_s, thr, P, hitmask);
-            __syncthreads();
+            if (kAhead) {
+                build_cluster(0);
+                if (nt > 1) build_cluster(1);
+                __syncthreads();
+            }
 
-            for (int j = 0; j < nt; ++j) {
-                const ProbeMeta m = meta[j];
-                const int pi = split + (t0 + j) * p.nsplit;
-                const int nblk = (m.len + kPointsPerBlock - 1) / kPointsPerBlock;
-                const uint4* cp = reinterpret_cast<const uint4*>(p.codes_il) + m.b0 * 32 + lane;
-                // The warp owns blocks warp, warp + 32, ...: `rem` of them are left, `ptr` is this lane's
-                // 16 bytes of the next one, `pos` the position of the lane's point in the list.  The
-                // first two blocks are requested now and needed after the table build.
-                constexpr int kStep = kWarps * 32;   // uint4 elements between two blocks of a warp
-                int rem = nblk > warp ? (nblk - warp + kWarps - 1) / kWarps : 0;
-                const uint4* ptr = cp + warp * 32;
-                int pos = warp * kPointsPerBlock + lane;
-                uint4 n0 = make_uint4(0, 0, 0, 0), n1 = make_uint4(0, 0, 0, 0);
-                if (rem > 0) n0 = __ldg(ptr);
-                if (rem > 1) n1 = __ldg(ptr + kStep);
-                // the warp's first blocks of the next list: into L2 while this list is scanned
-                if (kPf > 0 && j + 1 < nt) {
-                    const ProbeMeta m1 = meta[j + 1];
-                    const int nblk1 = (m1.len + kPointsPerBlock - 1) / kPointsPerBlock;
-                    const uint4* cp1 = reinterpret_cast<const uint4*>(p.codes_il) + m1.b0 * 32 + lane;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        if (warp + i * kWarps < nblk1) prefetch_l2(cp1 + (int64_t)(warp + i * kWarps) * 32);
-                }
-                // centroid of cluster j + 2 into the slot that the build of table j read
-                if (tid < 32 && j + 2 < nt) fetch_cent(meta[j + 2].cl, cent_s + (j & 1) * kD, tid);
-
-                if (DBG) {
-                    // masks of cluster j are complete (previous barrier); clear the other buffer
-                    if (p.masks)
-                        for (int i = tid; i < kW * 8; i += kNT)
-                            p.masks[(q * p.nprobe + pi) * kW * 8 + i] = hitmask[(j & 1) * kW * 8 + i];
-                    for (int i = tid; i < kW * 8; i += kNT) hitmask[((j + 1) & 1) * kW * 8 + i] = 0;
+            for (int j = 0; j < nt; j += 2) {
+                const bool two = j + 1 < nt;
+                if (!kAhead) {
+                    if (DBG && j > 0) {
+                        for (int i = tid; i < 2 * kW * 8; i += kNT) hitmask[i] = 0;
+                        __syncthreads();
+                    }
+                    // ---- phase A: the tables of clusters j and j + 1 ----
+                    build_cluster(j);
+                    if (two) build_cluster(j + 1);
                     __syncthreads();
                 }
-                // ---- this thread's share of the next cluster's table ----
-                if (j + 1 < nt)
-                    build(lut_gen + ((j + 1) & 1) * 128, cent_s + ((j + 1) & 1) * kD, thr, P, hitmask + ((j + 1) & 1) * kW * 8);
-
-                // ---- scan the list of cluster j (step D) ----
-                const uint32_t* hm = hitmask + (j & 1) * kW * 8;
+                if (DBG) {
+                    // the masks of this pair are complete (previous barrier)
+                    if (p.masks)
+                        for (int i = tid; i < (two ? 2 : 1) * kW * 8; i += kNT) {
+                            const int jj = j + i / (kW * 8);
+                            p.masks[(q * p.nprobe + split + (t0 + jj) * p.nsplit) * kW * 8 + i % (kW * 8)] =
+                                hitmask[(jj & (kSlots - 1)) * kW * 8 + i % (kW * 8)];
+                        }
+                    if (kAhead) {   // clear the buffers of the next pair before its tables are built
+                        for (int i = tid; i < 2 * kW * 8; i += kNT) hitmask[((j + 2) & 3) * kW * 8 + i] = 0;
+                        __syncthreads();
+                    }
+                }
+                // ---- scan the lists of clusters j and j + 1 (step D) ----
+                // Scan state of the list the warp is in: it owns blocks first, first + kWarps, ...:
+                // `rem` of them are left, `ptr` is this lane's 16 bytes of the next one, `pos` the
+                // position of the lane's point in the list; two blocks are always in registers.
+                constexpr int kStep = kWarps * 32;   // uint4 elements between two blocks of a warp
+                int li = 0, first = warp, pi = 0, rem = 0, pos = 0;
+                ProbeMeta m = meta[j];
+                const uint4* ptr = nullptr;
+                const uint32_t* hm = hitmask;
+                uint4 n0 = make_uint4(0, 0, 0, 0), n1 = make_uint4(0, 0, 0, 0);
+                auto enter = [&](int l) {
+                    m = meta[j + l];
+                    pi = split + (t0 + j + l) * p.nsplit;
+                    hm = hitmask + ((j + l) & (kSlots - 1)) * kW * 8;
+                    const int nblk = (m.len + kPointsPerBlock - 1) / kPointsPerBlock;
+                    rem = nblk > first ? (nblk - first + kWarps - 1) / kWarps : 0;
+                    ptr = reinterpret_cast<const uint4*>(p.codes_il) + m.b0 * 32 + lane + first * 32;
+                    pos = first * kPointsPerBlock + lane;
+                    if (rem > 0) n0 = __ldg(ptr);
+                    if (rem > 1) n1 = __ldg(ptr + kStep);
+                    // where the round-robin continues in the next list: the second list of the pair
+                    // goes on from this one's end, the next pair starts over
+                    const int next_first = l == 0 ? first + rem * kWarps - nblk : warp;
+                    if (kPf > 0 && j + l + 1 < nt) {   // the warp's first blocks of the next list: into L2 meanwhile
+                        const ProbeMeta m1 = meta[j + l + 1];
+                        const int nblk1 = (m1.len + kPointsPerBlock - 1) / kPointsPerBlock;
+                        const uint4* cp1 = reinterpret_cast<const uint4*>(p.codes_il) + m1.b0 * 32 + lane;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (next_first + i * kWarps < nblk1) prefetch_l2(cp1 + (int64_t)(next_first + i * kWarps) * 32);
+                    }
+                    first = next_first;
+                };
+                enter(0);   // the first two blocks are requested now and needed after the table build
+                if (kAhead) {
+                    // centroids of the pair after the next into the slots that the previous phase's
+                    // builds have read; this thread's share of the next pair's tables
+                    if (tid < 64 && j + 4 + (tid >> 5) < nt)
+                        fetch_cent(meta[j + 4 + (tid >> 5)].cl, cent_s + ((j + 4 + (tid >> 5)) & 3) * kD, lane);
+                    if (j + 2 < nt) build_cluster(j + 2);
+                    if (j + 3 < nt) build_cluster(j + 3);
+                } else {
+                    // centroids of the next pair into the slots that phase A has read
+                    if (tid < 64 && j + 2 + (tid >> 5) < nt)
+                        fetch_cent(meta[j + 2 + (tid >> 5)].cl, cent_s + (tid >> 5) * kD, lane);
+                }
                 while (true) {
                     const unsigned long long tau = *tau_p;
                     const uint32_t tau_hi = (uint32_t)(tau >> 32), tau_lo = (uint32_t)tau;
@@ -389,13 +437,21 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                             halt = __any_sync(0xFFFFFFFFu, stop);
                         }
                     };
-                    if (j & 1) scan_blocks(std::integral_constant<int, 1>{});
-                    else scan_blocks(std::integral_constant<int, 0>{});
+                    while (true) {
+                        const int table = (kAhead ? ((j >> 1) & 1) * 2 : 0) + li;
+                        if (table == 0) scan_blocks(std::integral_constant<int, 0>{});
+                        else if (table == 1) scan_blocks(std::integral_constant<int, 1>{});
+                        else if (kAhead && table == 2) scan_blocks(std::integral_constant<int, 2>{});
+                        else if (kAhead) scan_blocks(std::integral_constant<int, 3>{});
+                        if (halt || li == 1 || !two) break;
+                        li = 1;
+                        enter(1);
+                    }
                     cp_async_wait_all();
-                    // the barrier that separates cluster j from cluster j + 1 (table j + 1 complete,
-                    // table j free); a set flag means some warp saw the soft limit (it may have
-                    // finished its blocks all the same: the buffer is compacted before the next list)
-                    if (!__syncthreads_or(rem > 0 || halt)) break;
+                    // the barrier that ends the pair (tables free, next centroids staged); a set flag
+                    // means that some warp saw the soft limit or has blocks left: the buffer is
+                    // compacted and the scan resumes where it stopped
+                    if (!__syncthreads_or(rem > 0 || halt || (li == 0 && two))) break;
                     compact_candidates<kNT, kCap>(t, ntrans_p, hist_p, p.k, p.ids, kSoftLimit / 2);   // between lists any cut that frees half the buffer will do
                 }
             }
@@ -407,8 +463,9 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
 
 template <int NT, bool DBG, bool SCORED>
 cudaError_t launch_inst(const ScanParams& sp, int64_t grid, int64_t nitems, cudaStream_t st) {
-    // covers the table region (and the shared codebook of the 32-warp kernel) for any window offset
-    const size_t smem = NT == 1024 ? (size_t)kCbWin + 65536 : (size_t)kCbWin;
+    // covers, for any window offset, the auxiliary area, the table region and a second 64 KB region:
+    // the shared half of the codebook (32 warps) or the second pair of tables (16 warps)
+    const size_t smem = (size_t)kCbWin + 65536;
     auto kern = scan16x8_kernel<NT, DBG, SCORED>;
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
