@@ -10,16 +10,22 @@
 //     thread in registers, two in shared memory (two 16-byte loads per entry, conflict-free);
 //     eight warps per scheduler hide the latency of code blocks that stream from HBM: for long
 //     lists.  Either way building a table reads nothing from global memory but the probed centroid
-//     (512 B, copied two clusters ahead with cp.async).
+//     (512 B, copied one or two pairs of clusters ahead with cp.async).
 //   * Table layout: 256 rows (entries) of 256 bytes; a row holds two tables side by side, 32
 //     columns each; column x holds the value of subspace x & 15 (two copies).  Lane l looks up, at
 //     step i, column l ^ i: the 32 lanes of a warp touch 32 different banks whatever the codes
 //     are.  The code bytes are stored in that visiting order when the index is loaded.  The table
-//     region sits at shared-window address 0x10000, so one byte-permute forms the address (byte 0:
+//     regions sit at shared-window addresses 0x10000 (and 0x20000), so one byte-permute forms the address (byte 0:
 //     the lane's column offset for that step, byte 1: the code, bytes 2-3: zero) and the table base
 //     is the immediate of the load: three instructions per look-up.
-//   * Two tables: while the warps scan the list of cluster j they have already built their share of
-//     the table of cluster j + 1; one barrier per cluster separates the phases.
+//   * Clusters are taken two at a time and their two lists are dealt to the warps as one sequence
+//     of blocks, so that the barrier at the end of a phase waits for block counts that differ by
+//     one per pair of lists.  16 warps: four tables (a second 64 KB region); in one phase a warp
+//     builds its share of the next pair's tables and then scans this pair's lists - one barrier
+//     per pair.  32 warps (no room for four tables beside the shared codebook half): a phase that
+//     builds the pair's two tables, a phase that scans its lists.
+//   * The score (distance / count scores) is a template parameter: testing it for every table
+//     entry cost the distance search 9 %.
 //   * Code blocks: two per warp in registers, requested before the table build, refilled in
 //     two-block rounds without register copies; the 32-warp instance also asks for the lines
 //     further ahead to be brought into L2 (prefetch.global.L2, three blocks ahead and the first
