@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one scan-kernel launch, from the ncu captures
 # summarised under profiles/ (bytes per launch of the benchmark's workload; None = not captured).
-SCAN_DRAM_TRAFFIC_BYTES = {"c2": 26.6e6, "c5": 72.5e9}
+SCAN_DRAM_TRAFFIC_BYTES = {"c2": 26.6e6, "c5": 72.2e9}
 
 
 def log(*a):
