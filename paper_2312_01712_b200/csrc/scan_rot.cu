@@ -214,8 +214,10 @@ template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, bool SCORED>
 __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const ScanParams p) {
     using GR = Groups<W0, W1, W2>;
     constexpr int kWarps = NT / 32;
-    constexpr int kBlocksPerWarpRound = 1024 / NT;       // 1024 candidates per round, CTA-wide
-    static_assert(IVFPQ_MAX_K + 1024 <= kTopkCap, "candidate buffer too small for a round");
+    // A warp stops after the block in which one of its candidates landed at or beyond the soft limit
+    // (at most 32 more per warp): the buffer is then reduced to the k smallest at the next barrier.
+    constexpr int kSoft = kTopkCap - 32 * kWarps;
+    static_assert(IVFPQ_MAX_K < kSoft, "candidate buffer too small for the soft limit");
     extern __shared__ __align__(16) unsigned char smem[];
     const int nsub = GR::kNsub;
     const int ksub = p.ksub;
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
             if (tid == 0) atomicOr(p.status, kFlagBadList);
             continue;
         }
-        __syncthreads();  // the previous cluster's scan no longer reads the tables
+        // (the barrier that ended the previous cluster's scan makes the tables and `res` free)
         for (int j = tid; j < d; j += NT) res[j] = __fsub_rn(p.queries[q * d + j], p.cent[(int64_t)c * d + j]);
         if (DBG)
             for (int i = tid; i < IVFPQ_MAX_NSUB * 8; i += NT) hitmask[i] = 0;
@@ -325,13 +327,14 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
             continue;
         }
         const unsigned char* cbase = reinterpret_cast<const unsigned char*>(p.codes_il) + b0 * GR::kBlockBytes;
-        for (int64_t bb = 0; bb < nblk; bb += kWarps * kBlocksPerWarpRound) {
+        int64_t blk = warp;   // the warp scans blocks warp, warp + kWarps, ...
+        while (true) {
             const unsigned long long tau = *tau_p;
             const uint32_t tau_hi = (uint32_t)(tau >> 32);
+            bool halt = false;
 #pragma unroll 1
-            for (int r = 0; r < kBlocksPerWarpRound; ++r) {
-                const int64_t blk = bb + r * kWarps + warp;
-                if (blk >= nblk) break;
+            for (; blk < nblk && !halt; blk += kWarps) {
+                bool stop = false;
                 const unsigned char* bp = cbase + blk * GR::kBlockBytes;
                 uint32_t w0[W0 >= 4 ? W0 / 4 : 1];
                 uint32_t w1[W1 >= 4 ? W1 / 4 : 1];
@@ -369,12 +372,20 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
                     if (__float_as_uint(acc) <= tau_hi) {
                         const unsigned long long key = make_key(acc, (uint32_t)p.ids[p0 + pos]);
                         if (key < tau) {
-                            if (!topk_push(t, key)) atomicOr(p.status, kFlagOverflow);
+                            const int slot = atomicAdd(cnt_p, 1);
+                            if (slot < kTopkCap) kbuf[slot] = key;
+                            else atomicOr(p.status, kFlagOverflow);
+                            stop = slot >= kSoft;
                         }
                     }
                 }
+                halt = __any_sync(0xFFFFFFFFu, stop);
             }
-            topk_round_end<NT>(t, p.k, 1024);
+            // The barrier that ends the cluster (tables free for the next one).  A set flag means that a
+            // warp met the soft limit (it may have finished its blocks all the same): the buffer is
+            // reduced to the k smallest keys and the scan resumes where it stopped.
+            if (!__syncthreads_or(blk < nblk || halt)) break;
+            topk_select<NT>(t, p.k);
         }
     }
 
