@@ -342,18 +342,24 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
     if (!all_exact) {
         // ---- a bound at or above the nprobe-th smallest approximate distance: stream the row
         //      through the buffer, compacting by histogram whenever it could overflow ----
-        for (int base = 0; base < nlist; base += 256) {
-            const int c = base + tid;
-            if (c < nlist) {
-                const unsigned long long key = make_key(fmaxf(row[c] + qn, 0.0f), (uint32_t)c);
-                if (key < tau) {
-                    if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
+        if (nlist <= kTopkCap) {
+            // the whole row fits the buffer: every key goes to its own slot, no counting, no barriers
+            for (int c = tid; c < nlist; c += 256) buf[c] = make_key(fmaxf(row[c] + qn, 0.0f), (uint32_t)c);
+            if (tid == 0) cnt = nlist;
+        } else {
+            for (int base = 0; base < nlist; base += 256) {
+                const int c = base + tid;
+                if (c < nlist) {
+                    const unsigned long long key = make_key(fmaxf(row[c] + qn, 0.0f), (uint32_t)c);
+                    if (key < tau) {
+                        if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
+                    }
                 }
+                __syncthreads();
+                const int filled = cnt;
+                __syncthreads();
+                if (filled + 256 > kTopkCap) topk_quick_compact<256>(t, nprobe, hist);
             }
-            __syncthreads();
-            const int filled = cnt;
-            __syncthreads();
-            if (filled + 256 > kTopkCap) topk_quick_compact<256>(t, nprobe, hist);
         }
         topk_quick_compact<256>(t, nprobe, hist);   // starts and ends with a barrier
         const float bound = __uint_as_float((uint32_t)(tau >> 32));   // every kept key is below it; +inf when nothing was dropped
