@@ -129,9 +129,11 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
 
 WorkspaceLayout plan_workspace(const ivfpq_index* ix, int64_t nq, int32_t nprobe, int32_t k) {
     WorkspaceLayout wl{};
-    // query chunk of the filtering stage: keep the [qchunk][nlist] distance tile near 32 MiB so
-    // that it stays in L2 between the kernel that writes it and the one that selects from it
-    int64_t qchunk = ((int64_t)32 << 20) / ((int64_t)ix->nlist * 4);
+    // query chunk of the filtering stage: keep the [qchunk][nlist] distance tile near 64 MiB, so
+    // that it stays in the 126 MB L2 between the kernel that writes it and the one that selects
+    // from it, with as many queries per launch as that allows (measured: 32 MiB and 96 MiB are
+    // both slower on the 16 384-cluster workload)
+    int64_t qchunk = ((int64_t)64 << 20) / ((int64_t)ix->nlist * 4);
     if (qchunk < 64) qchunk = 64;
     if (qchunk > nq) qchunk = nq;
     wl.qchunk = qchunk;

@@ -93,6 +93,24 @@ def test_probe_lists_tensor_core_shapes():
         lib.ivfpq_index_free(h)
 
 
+def test_probe_lists_many_clusters():
+    """More clusters than the exact decision's candidate buffer holds (the row of approximate
+    distances is streamed through it in batches), small and large probe counts."""
+    wl = Workload(small_cfg("c1", n=24_000, d=64, nsub=8, dsub=8, ncomp=400, nlist=5000, nq=150, chunk=16384,
+                            kmeans_iters=2))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        q = dev(wl.queries)
+        for nprobe in (1, 32, 300, 1024):
+            pid, pd = lib.ivfpq_debug_probes(h, q, nprobe)
+            opid, opd = oracle.coarse(wl.index, wl.queries, nprobe)
+            check_status(h)
+            assert np.array_equal(host(pid), opid)
+            assert np.array_equal(host(pd).view(np.uint32), opd.view(np.uint32))
+    finally:
+        lib.ivfpq_index_free(h)
+
+
 def test_probe_all_lists(loaded):
     wl, h = loaded["small"]
     pid, pd = lib.ivfpq_debug_probes(h, dev(wl.queries), wl.index.nlist)
