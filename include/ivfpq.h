@@ -199,7 +199,14 @@ int ivfpq_search_sparse(const ivfpq_index_t* index, const float* queries, int64_
  * queries to the device, search, copy distances and ids back, all enqueued on `stream`.  The
  * staging areas live in the caller's workspace, whose size is given by
  * ivfpq_search_host_workspace_bytes.  `radius` (NULL = dense search) still points to a struct
- * whose `radius` array is device memory. */
+ * whose `radius` array is device memory.
+ * Batches of 2048 queries or more are processed in two slices: a copy stream that the
+ * handle creates on first use (with a few events: host-side resources, no device memory) brings
+ * the slices' queries in and takes the first slice's results out while `stream` searches the
+ * second.  Everything is ordered with respect to `stream`: work enqueued on it after this call
+ * sees the results in the host buffers; the device status word covers all slices.  Use pinned
+ * host buffers for the copies to overlap.  Calls on one handle must not be issued from several
+ * host threads at once. */
 size_t ivfpq_search_host_workspace_bytes(const ivfpq_index_t* index, int64_t nq, int32_t nprobe, int32_t k);
 int ivfpq_search_host(const ivfpq_index_t* index, const float* queries_host, int64_t nq, int32_t nprobe,
                       const ivfpq_radius_t* radius, int32_t k, float* out_dist_host,

@@ -70,7 +70,8 @@ int check_search_shape(const ivfpq_index* ix, int64_t nq, int32_t nprobe, int32_
     return IVFPQ_OK;
 }
 
-int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stream, bool probes_only) {
+int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stream, bool probes_only,
+               bool keep_status = false) {
     const ivfpq_index* ix = a.ix;
     int rc = check_search_shape(ix, a.nq, a.nprobe, a.k);
     if (rc != IVFPQ_OK) return rc;
@@ -96,7 +97,8 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
             if (cudaEventCreate(&ix->ev[i]) != cudaSuccess) return IVFPQ_ERR_CUDA;
         ix->ev_ready = true;
     }
-    if (cudaMemsetAsync(ws + wl.status_off, 0, 16, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    // keep_status: a later slice of one batch adds its flags to those of the earlier slices
+    if (!keep_status && cudaMemsetAsync(ws + wl.status_off, 0, 16, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
     if (timed && cudaEventRecord(ix->ev[0], st) != cudaSuccess) return IVFPQ_ERR_CUDA;
     int32_t* probe_ids = reinterpret_cast<int32_t*>(ws + wl.probe_ids_off);
     float* probe_d = reinterpret_cast<float*>(ws + wl.probe_d_off);
@@ -234,6 +236,7 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->last_launches = 0;
     ix->timing = 0;
     ix->ev_ready = false;
+    ix->pipe_ready = false;
     ix->ev_recorded = false;
 
     // list tables: built on the host, copied synchronously (pageable source)
@@ -270,6 +273,10 @@ int ivfpq_index_free(ivfpq_index_t* index) {
     if (!index) return IVFPQ_ERR_INVALID_ARGUMENT;
     if (index->ev_ready)
         for (int i = 0; i < 3; ++i) cudaEventDestroy(index->ev[i]);
+    if (index->pipe_ready) {
+        for (int i = 0; i < 12; ++i) cudaEventDestroy(index->pipe_ev[i]);
+        cudaStreamDestroy(index->copy_stream);
+    }
     delete index;
     return IVFPQ_OK;
 }
@@ -371,8 +378,6 @@ int ivfpq_search_host(const ivfpq_index_t* index, const float* queries_host, int
     off = align_up(off + (size_t)nq * k * 4, 256);
     int32_t* i_dev = reinterpret_cast<int32_t*>(ws + off);
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(q_dev, queries_host, (size_t)nq * index->d * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return IVFPQ_ERR_CUDA;
     SearchArgs a{};
     a.ix = index;
     a.queries = q_dev;
@@ -383,6 +388,57 @@ int ivfpq_search_host(const ivfpq_index_t* index, const float* queries_host, int
     if (radius) fill_radius(a, radius);
     a.out_dist = d_dev;
     a.out_ids = i_dev;
+
+    // Large batches go in slices: the copy stream brings all slices' queries in and takes each
+    // slice's results out while the caller's stream searches the next slice.  (With the stage
+    // timing option on, the batch stays in one piece so that the stage times describe it.)
+    // (measured on the 10 k-query batch: two slices +2.4 % end to end, three +1.9 %, four none)
+    const int nslice = index->timing ? 1 : (nq >= 2048 ? 2 : 1);
+    if (nslice > 1) {
+        if (!index->pipe_ready) {
+            if (cudaStreamCreateWithFlags(&index->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return IVFPQ_ERR_CUDA;
+            for (int i = 0; i < 12; ++i)
+                if (cudaEventCreateWithFlags(&index->pipe_ev[i], cudaEventDisableTiming) != cudaSuccess) return IVFPQ_ERR_CUDA;
+            index->pipe_ready = true;
+        }
+        cudaStream_t cs = index->copy_stream;
+        cudaEvent_t* ev = index->pipe_ev;   // [0]: start, [1 + s]: queries of slice s in, [5 + s]: slice s searched, [9]: all out
+        const int64_t per = ((nq + nslice - 1) / nslice + 31) / 32 * 32;
+        bool ok = cudaEventRecord(ev[0], st) == cudaSuccess && cudaStreamWaitEvent(cs, ev[0], 0) == cudaSuccess;
+        for (int s = 0; ok && s < nslice; ++s) {
+            const int64_t lo = s * per, n = lo < nq ? (nq - lo < per ? nq - lo : per) : 0;
+            if (n <= 0) continue;
+            ok = cudaMemcpyAsync(q_dev + lo * index->d, queries_host + lo * index->d, (size_t)n * index->d * 4,
+                                 cudaMemcpyHostToDevice, cs) == cudaSuccess &&
+                 cudaEventRecord(ev[1 + s], cs) == cudaSuccess;
+        }
+        if (!ok) return IVFPQ_ERR_CUDA;
+        int64_t launches = 0;
+        for (int s = 0; s < nslice; ++s) {
+            const int64_t lo = s * per, n = lo < nq ? (nq - lo < per ? nq - lo : per) : 0;
+            if (n <= 0) continue;
+            if (cudaStreamWaitEvent(st, ev[1 + s], 0) != cudaSuccess) return IVFPQ_ERR_CUDA;
+            SearchArgs b = a;
+            b.queries = q_dev + lo * index->d;
+            b.nq = n;
+            b.out_dist = d_dev + lo * k;
+            b.out_ids = i_dev + lo * k;
+            if (!b.dense && b.radius_mode == 1) b.radius = a.radius + lo * index->nsub;
+            rc = run_search(b, workspace, core, stream, false, s > 0);
+            if (rc != IVFPQ_OK) return rc;
+            launches += index->last_launches;
+            ok = cudaEventRecord(ev[5 + s], st) == cudaSuccess && cudaStreamWaitEvent(cs, ev[5 + s], 0) == cudaSuccess &&
+                 cudaMemcpyAsync(out_dist_host + lo * k, d_dev + lo * k, (size_t)n * k * 4, cudaMemcpyDeviceToHost, cs) == cudaSuccess &&
+                 cudaMemcpyAsync(out_ids_host + lo * k, i_dev + lo * k, (size_t)n * k * 4, cudaMemcpyDeviceToHost, cs) == cudaSuccess;
+            if (!ok) return IVFPQ_ERR_CUDA;
+        }
+        index->last_launches = launches;
+        if (cudaEventRecord(ev[9], cs) != cudaSuccess || cudaStreamWaitEvent(st, ev[9], 0) != cudaSuccess) return IVFPQ_ERR_CUDA;
+        return IVFPQ_OK;
+    }
+
+    if (cudaMemcpyAsync(q_dev, queries_host, (size_t)nq * index->d * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
     rc = run_search(a, workspace, core, stream, false);
     if (rc != IVFPQ_OK) return rc;
     if (cudaMemcpyAsync(out_dist_host, d_dev, (size_t)nq * k * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)

@@ -54,6 +54,11 @@ struct ivfpq_index {
     int32_t timing;           // IVFPQ_OPT_TIMING
     mutable cudaEvent_t ev[3];  // start, after filtering, end (created lazily)
     mutable bool ev_ready, ev_recorded;
+    // host entry point: a copy stream and events that let the transfers of one slice of the batch
+    // overlap with the search of another (created on first use)
+    mutable cudaStream_t copy_stream;
+    mutable cudaEvent_t pipe_ev[12];
+    mutable bool pipe_ready;
 };
 
 namespace ivfpq {

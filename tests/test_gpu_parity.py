@@ -328,6 +328,40 @@ def test_host_buffer_entry_point_matches_device_entry_point(loaded):
     assert np.array_equal(od.numpy(), host(d)) and np.array_equal(oi.numpy(), host(i))
 
 
+@pytest.mark.parametrize("nq", [2048, 5003])
+def test_host_entry_point_in_slices(loaded, nq):
+    """Large batches go through the host entry point in slices (transfers of one slice overlap
+    the search of another): same results as one device call, per-query radii follow their slice,
+    the status covers every slice."""
+    wl, h = loaded["small"]
+    rng = np.random.default_rng(nq)
+    pick = rng.integers(0, wl.queries.shape[0], nq)
+    q = np.ascontiguousarray(wl.queries[pick] + rng.standard_normal((nq, wl.queries.shape[1])).astype(F32) * 0.01)
+    rad = np.ascontiguousarray(wl.radius_per_query[pick] * (1 + 0.1 * rng.random((nq, wl.index.nsub), dtype=F32)))
+    k = 25
+    qh = torch.from_numpy(q).pin_memory()
+    od = torch.empty((nq, k), dtype=torch.float32).pin_memory()
+    oi = torch.empty((nq, k), dtype=torch.int32).pin_memory()
+    for radius in (None, dev(rad), dev(wl.radius)):
+        od.fill_(-1.0)
+        oi.fill_(-7)
+        lib.ivfpq_search_host(h, qh, 5, k, od, oi, radius=radius, scale=0.9)
+        check_status(h)   # synchronises the stream
+        if radius is None:
+            d, i = lib.ivfpq_search_dense(h, dev(q), 5, k)
+        else:
+            d, i = lib.ivfpq_search_sparse(h, dev(q), 5, radius, k, scale=0.9)
+        check_status(h)
+        assert np.array_equal(oi.numpy(), host(i))
+        assert np.array_equal(od.numpy().view(np.uint32), host(d).view(np.uint32))
+    # against the oracle on a sample, and a bad probe count still fails up front
+    sel = np.sort(rng.choice(nq, 64, replace=False))
+    o = oracle.search(wl.index, q[sel], 5, k, radius=wl.radius, scale=0.9)
+    assert_topk_parity(od.numpy()[sel], oi.numpy()[sel], o["dist"], o["ids"])
+    with pytest.raises(lib.IvfpqError):
+        lib.ivfpq_search_host(h, qh, wl.index.nlist + 1, k, od, oi)
+
+
 def test_error_codes_on_gpu(loaded):
     wl, h = loaded["small"]
     q = dev(wl.queries)
