@@ -24,8 +24,8 @@
 //     builds its share of the next pair's tables and then scans this pair's lists - one barrier
 //     per pair.  32 warps (no room for four tables beside the shared codebook half): a phase that
 //     builds the pair's two tables, a phase that scans its lists.
-//   * The score (distance / count scores) is a template parameter: testing it for every table
-//     entry cost the distance search 9 %.
+//   * The score (distance / hit count / reward-penalty) is a template parameter: testing it for
+//     every table entry cost the distance search 9 %.
 //   * Code blocks: two per warp in registers, requested before the table build, refilled in
 //     two-block rounds without register copies; the 32-warp instance also asks for the lines
 //     further ahead to be brought into L2 (prefetch.global.L2, three blocks ahead and the first
@@ -108,7 +108,7 @@ __device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[
     return a0 + a1;
 }
 
-template <int NT, bool DBG, bool SCORED>
+template <int NT, bool DBG, int SCORE_T>
 __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, const int64_t nitems) {
     constexpr int kNT = NT;
     constexpr int kWarps = Shape<NT>::kWarps;
@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
             }
             const int e = u + kEP * m;
             const bool hit = e < ksub && (p.dense || d2 <= thr);
-            const float val = table_value<SCORED>(p.score, hit, d2, thr, P);
+            const float val = table_value<SCORE_T>(p.score, hit, d2, thr, P);
             unsigned char* row = lutb + m * (kEP * kRowBytes);
             *reinterpret_cast<float*>(row + st_a) = val;
             *reinterpret_cast<float*>(row + st_b) = val;
@@ -467,24 +467,25 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
     }
 }
 
-template <int NT, bool DBG, bool SCORED>
+template <int NT, bool DBG, int SCORE_T>
 cudaError_t launch_inst(const ScanParams& sp, int64_t grid, int64_t nitems, cudaStream_t st) {
     // covers, for any window offset, the auxiliary area, the table region and a second 64 KB region:
     // the shared half of the codebook (32 warps) or the second pair of tables (16 warps)
     const size_t smem = (size_t)kCbWin + 65536;
-    auto kern = scan16x8_kernel<NT, DBG, SCORED>;
+    auto kern = scan16x8_kernel<NT, DBG, SCORE_T>;
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<(unsigned)grid, NT, smem, st>>>(sp, nitems);
     return cudaGetLastError();
 }
 
-// Instances: stage dumps (any score), count scores, distances only (the benchmarked path).
+// Instances: stage dumps (score read at run time), one per score otherwise.
 template <int NT>
 cudaError_t launch_nt(const ScanParams& sp, int64_t grid, int64_t nitems, bool debug, cudaStream_t st) {
-    if (debug) return launch_inst<NT, true, true>(sp, grid, nitems, st);
-    if (sp.score != IVFPQ_SCORE_DISTANCE) return launch_inst<NT, false, true>(sp, grid, nitems, st);
-    return launch_inst<NT, false, false>(sp, grid, nitems, st);
+    if (debug) return launch_inst<NT, true, -1>(sp, grid, nitems, st);
+    if (sp.score == IVFPQ_SCORE_HIT_COUNT) return launch_inst<NT, false, IVFPQ_SCORE_HIT_COUNT>(sp, grid, nitems, st);
+    if (sp.score == IVFPQ_SCORE_REWARD_PENALTY) return launch_inst<NT, false, IVFPQ_SCORE_REWARD_PENALTY>(sp, grid, nitems, st);
+    return launch_inst<NT, false, IVFPQ_SCORE_DISTANCE>(sp, grid, nitems, st);
 }
 
 }  // namespace

@@ -45,13 +45,15 @@ struct ScanParams {
 // squared distance, or the miss constant P (paper Sec. 5.3).  Count scores (Sec. 5.4): 0 / 1 for
 // selected / not selected; with the inner sphere of half the radius 0 / 1 / 2 for inside the inner
 // sphere / between the two / outside both.  The list scan sums slots, whatever they hold.
-// SCORED = false: a kernel instance that serves distances only.  The choice is made per launch, not
-// per entry: with the score tested for every entry the table build of the 16 x 8 kernel cost 9 % of
-// the whole search, that of the 50 x 4 kernel 15 %.
-template <bool SCORED = true>
+// SCORE_T >= 0: a kernel instance compiled for that score; SCORE_T < 0: the score is read at run time
+// (stage-dump instances, generic kernel).  The choice is made per launch, not per entry: with the
+// score tested for every entry the table build of the 16 x 8 kernel cost 9 % of the whole search,
+// that of the 50 x 4 kernel 15 %.
+template <int SCORE_T = -1>
 __device__ __forceinline__ float table_value(int score, bool hit, float d2, float thr, float P) {
-    if (!SCORED || score == IVFPQ_SCORE_DISTANCE) return hit ? d2 : P;
-    if (score == IVFPQ_SCORE_HIT_COUNT) return hit ? 0.0f : 1.0f;
+    const int sc = SCORE_T >= 0 ? SCORE_T : score;
+    if (sc == IVFPQ_SCORE_DISTANCE) return hit ? d2 : P;
+    if (sc == IVFPQ_SCORE_HIT_COUNT) return hit ? 0.0f : 1.0f;
     return !hit ? 2.0f : (d2 <= __fmul_rn(0.25f, thr) ? 0.0f : 1.0f);
 }
 

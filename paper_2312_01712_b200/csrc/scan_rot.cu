@@ -77,7 +77,7 @@ __host__ __device__ inline size_t rot_smem_bytes(bool paired, int lut_floats, in
 
 // Table of one group for one (query, cluster): thread t owns column c = t & (W-1) and the
 // entries u, u + NT/W, ... with u = t / W.
-template <int W, int DSUB, int NT, bool DBG, bool SCORED, int RS = row_stride(W)>
+template <int W, int DSUB, int NT, bool DBG, int SCORE_T, int RS = row_stride(W)>
 __device__ __forceinline__ void build_group(float* __restrict__ lutg, const float* __restrict__ cbt_g,
                                             const float* __restrict__ res_g, const float* __restrict__ r2_g,
                                             int ksub, bool dense, int score, float P, uint32_t* hitmask_g) {
@@ -124,7 +124,7 @@ __device__ __forceinline__ void build_group(float* __restrict__ lutg, const floa
             }
             hit = dense || d2 <= thr;
         }
-        const float val = table_value<SCORED>(score, hit, d2, thr, P);
+        const float val = table_value<SCORE_T>(score, hit, d2, thr, P);
         float* row = lutg + e * RS + c;
 #pragma unroll
         for (int it = 0; it < NCOPY; ++it) {
@@ -210,7 +210,7 @@ __device__ __forceinline__ void load_group_codes(const unsigned char* __restrict
     }
 }
 
-template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, bool SCORED>
+template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T>
 __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const ScanParams p) {
     using GR = Groups<W0, W1, W2>;
     constexpr int kWarps = NT / 32;
@@ -304,13 +304,13 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
         __syncthreads();
 
         // ---- selective tables, one per group ----
-        build_group<W0, DSUB, NT, DBG, SCORED, GR::stride(0)>(lut, p.cbt, res, r2, ksub, p.dense, p.score, P, hitmask);
+        build_group<W0, DSUB, NT, DBG, SCORE_T, GR::stride(0)>(lut, p.cbt, res, r2, ksub, p.dense, p.score, P, hitmask);
         if constexpr (W1 > 0)
-            build_group<W1, DSUB, NT, DBG, SCORED, GR::stride(1)>(lut + GR::lut_off(1), p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
+            build_group<W1, DSUB, NT, DBG, SCORE_T, GR::stride(1)>(lut + GR::lut_off(1), p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
                                            res + GR::s0(1) * DSUB, r2 + GR::s0(1), ksub, p.dense, p.score, P,
                                            hitmask + GR::s0(1) * 8);
         if constexpr (W2 > 0)
-            build_group<W2, DSUB, NT, DBG, SCORED>(lut + GR::lut_off(2), p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
+            build_group<W2, DSUB, NT, DBG, SCORE_T>(lut + GR::lut_off(2), p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
                                            res + GR::s0(2) * DSUB, r2 + GR::s0(2), ksub, p.dense, p.score, P,
                                            hitmask + GR::s0(2) * 8);
         __syncthreads();
@@ -403,22 +403,25 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
     }
 }
 
-template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, bool SCORED>
+template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T>
 cudaError_t launch_rot_inst(const ScanParams& sp, int64_t grid, int nprobe, cudaStream_t st) {
     const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kPaired, Groups<W0, W1, W2>::kLutFloats, sp.d, nprobe, DBG);
-    auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, DBG, SCORED>;
+    auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, DBG, SCORE_T>;
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<(unsigned)grid, NT, smem, st>>>(sp);
     return cudaGetLastError();
 }
 
-// Instances: stage dumps (any score), count scores, distances only.
+// Instances: stage dumps (score read at run time), one per score otherwise.
 template <int W0, int W1, int W2, int DSUB, int NT>
 cudaError_t launch_rot(const ScanParams& sp, int64_t grid, bool debug, int nprobe, cudaStream_t st) {
-    if (debug) return launch_rot_inst<W0, W1, W2, DSUB, NT, true, true>(sp, grid, nprobe, st);
-    if (sp.score != IVFPQ_SCORE_DISTANCE) return launch_rot_inst<W0, W1, W2, DSUB, NT, false, true>(sp, grid, nprobe, st);
-    return launch_rot_inst<W0, W1, W2, DSUB, NT, false, false>(sp, grid, nprobe, st);
+    if (debug) return launch_rot_inst<W0, W1, W2, DSUB, NT, true, -1>(sp, grid, nprobe, st);
+    if (sp.score == IVFPQ_SCORE_HIT_COUNT)
+        return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_HIT_COUNT>(sp, grid, nprobe, st);
+    if (sp.score == IVFPQ_SCORE_REWARD_PENALTY)
+        return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_REWARD_PENALTY>(sp, grid, nprobe, st);
+    return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_DISTANCE>(sp, grid, nprobe, st);
 }
 
 }  // namespace
