@@ -466,6 +466,14 @@ def run_reference(args):
     k = cfg.k
     sample = min(args.cpu_sample, q_np.shape[0])
     scale = args.ref_scale
+    if scale <= 0:
+        # the same rule as the CUDA arm (smallest scale whose recall@100 is within 0.01 of dense),
+        # decided by the oracle on the first 1000 queries
+        ns = min(1000, q_np.shape[0])
+        _, _, (scale, _, _), sweep = pick_scale(
+            lambda sc: oracle.search(index, q_np[:ns], nprobe, k, radius=radius, scale=sc)["ids"],
+            lambda: oracle.search(index, q_np[:ns], nprobe, k, dense=True)["ids"], true_ids[:ns])
+        log(f"[bench] reference arm: radius scale {scale} (sweep {sweep})")
     for _ in range(min(args.warmup, 1)):
         oracle.search(index, q_np[:64], nprobe, k, radius=radius, scale=scale)
     steps = min(args.steps, 5)
@@ -500,7 +508,8 @@ def main():
     ap.add_argument("--nprobe", type=int, default=0)
     ap.add_argument("--nq", type=int, default=None)
     ap.add_argument("--cpu-sample", type=int, default=10000, help="queries timed on the CPU oracle")
-    ap.add_argument("--ref-scale", type=float, default=1.0)
+    ap.add_argument("--ref-scale", type=float, default=0.0,
+                    help="radius scale of the reference arm; 0 = chosen by the CUDA arm's recall rule")
     ap.add_argument("--dynamic-radius", action="store_true",
                     help="query-specific thresholds from density maps + polynomial regressor (workload c3)")
     ap.add_argument("--metric", default="l2", choices=["l2", "ip"],
