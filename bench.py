@@ -6,7 +6,7 @@ construction, list scan, top-k - over one batch of synthetic queries through the
 ABI (`ivfpq_search_sparse` at the radius scale whose recall@100 is within 0.01 of
 the dense search).  Prints ONE JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--nprobe 16]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--nprobe 32]
     python bench.py --impl reference ...      # the CPU oracle on the host cores
 
 Multi-GPU (torchrun, one rank per GPU): the index is replicated and every rank
@@ -40,9 +40,11 @@ METRIC = "queries/sec at recall@100 (1 B200) + scan HBM GB/s as % of peak"
 UNIT = "queries/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one scan-kernel launch, from the ncu captures
-# summarised under profiles/ (bytes per launch of the benchmark's workload; None = not captured).
-SCAN_DRAM_TRAFFIC_BYTES = {"c2": 26.6e6, "c5": 72.2e9}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel at the default
+# settings of a workload, from the ncu capture summarised in the named file under profiles/ (taken
+# on a smaller query batch and scaled by the points visited).  An entry is dropped (traffic: null)
+# when the kernel it describes changes.
+SCAN_DRAM_TRAFFIC = {}
 
 
 def log(*a):
@@ -227,6 +229,34 @@ def visits_per_batch(index, probe_ids: np.ndarray) -> int:
     return int(lens[probe_ids].sum())
 
 
+def selection_stats(lib, h, index, qd, nprobe, k, rad_d, scale, score, sample=16):
+    """What the selection does at this radius scale, from the stage dumps of a small query sample
+    (outside any timed region): the mean fraction of codebook entries selected per (query, probed
+    cluster, subspace), the fraction of visited points whose entry was selected in every subspace,
+    and the mean fraction of subspaces selected per visited point."""
+    n = min(sample, qd.shape[0])
+    qs = qd[:n].contiguous()
+    rad = rad_d if rad_d.dim() == 1 else rad_d[:n].contiguous()
+    probe_ids = lib.ivfpq_debug_probes(h, qs, nprobe)[0].cpu().numpy()
+    lens = np.diff(index.list_offsets)
+    stride = int(lens[probe_ids].sum(axis=1).max())
+    r = lib.ivfpq_debug_search(h, qs, nprobe, k, radius=rad, scale=scale, visit_stride=stride, score=score)
+    masks = r["masks"].cpu().numpy().view(np.uint32)
+    sel = float(np.unpackbits(masks.view(np.uint8)).sum()) / (masks.shape[0] * masks.shape[1] * index.nsub * index.ksub)
+    vcount = r["visit_count"].cpu().numpy()
+    hits = r["visit_hits"].cpu().numpy().view(np.uint64)
+    full = np.uint64((1 << index.nsub) - 1)
+    allhit = nvis = nbits = 0
+    for i in range(n):
+        hrow = hits[i, :vcount[i]]
+        allhit += int((hrow == full).sum())
+        nbits += int(np.unpackbits(hrow.view(np.uint8)).sum())
+        nvis += int(vcount[i])
+    return {"queries_sampled": n, "selected_entry_fraction": round(sel, 4),
+            "all_hit_point_fraction": round(allhit / max(1, nvis), 5),
+            "selected_subspaces_per_point": round(nbits / max(1, nvis) / index.nsub, 4)}
+
+
 # --------------------------------------------------------------------------------------------
 # the CUDA arm
 # --------------------------------------------------------------------------------------------
@@ -286,6 +316,8 @@ def run_cuda(args):
     assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
     log(f"[bench] recall@100 dense {r_dense:.4f}, sparse {r_sparse:.4f} at scale {scale} (sweep {sweep})")
 
+    sel_stats = selection_stats(lib, h, index, qd, nprobe, k, rad_d, scale, score)
+    log(f"[bench] selection at scale {scale}: {sel_stats}")
     probe_ids = lib.ivfpq_debug_probes(h, qd, nprobe)[0].cpu().numpy()
     visits = visits_per_batch(index, probe_ids)
     scan_bytes = visits * index.nsub          # algorithmic: one code byte per subspace per visited point
@@ -378,12 +410,33 @@ def run_cuda(args):
         peak, peak_src = FALLBACK_HBM_GBS, "fallback"
     scan_ms = float(np.mean([s[1] for s in stages]))
     coarse_ms = float(np.mean([s[0] for s in stages]))
-    achieved = scan_bytes / (scan_ms * 1e-3) / 1e9
-    # shared-memory ceiling of the scan: one conflict-free 32-lane table gather per SM per clock
     props = torch.cuda.get_device_properties(local_rank)
     clk = sampler.summary()["sm_mhz"] or sampler.summary()["sm_max_mhz"] or 1965.0
+    # Which ceiling binds the list scan depends on where the codes live.  Larger than the L2 cache:
+    # the scan streams them from HBM, algorithmic bytes = one code byte per subspace per visited
+    # point.  Inside the L2 cache: DRAM sees next to nothing and the ceiling is the shared-memory
+    # table gather (one conflict-free 32-lane gather per SM per clock, one gather per code byte).
+    code_bytes_total = int(index.ntotal) * index.nsub
+    l2_bytes = int(getattr(props, "L2_cache_size", 126 << 20))
+    hbm_gbs = scan_bytes / (scan_ms * 1e-3) / 1e9
     gather_peak = props.multi_processor_count * 32 * clk * 1e6 / 1e9            # G gathers/s
-    gather_rate = scan_bytes / (scan_ms * 1e-3) / 1e9                            # one gather per code byte
+    kernel = scan_kernel_name(index) + " (selective LUT + list scan + top-k)"
+    default_run = args.nq is None and args.nprobe == 0 and score == 0 and metric == 0 and not dynamic
+    traffic = SCAN_DRAM_TRAFFIC.get(args.workload) if default_run else None
+    common = {"kernel": kernel, "algorithmic_bytes_per_launch": int(scan_bytes), "visits_per_launch": int(visits),
+              "kernel_ms": scan_ms, "traffic": traffic,
+              "codes": f"{code_bytes_total / 1e6:.0f} MB of codes against {l2_bytes / 1e6:.0f} MB of L2"}
+    if code_bytes_total > l2_bytes:
+        roofline = {"bound": "hbm", "achieved": hbm_gbs, "peak": peak, "unit": "GB/s", "frac": hbm_gbs / peak,
+                    "peak_source": f"of {peak_src}", **common,
+                    "gather_frac": hbm_gbs / gather_peak}
+    else:
+        roofline = {"bound": "shared-memory gathers", "achieved": hbm_gbs, "peak": gather_peak, "unit": "Ggather/s",
+                    "frac": hbm_gbs / gather_peak,
+                    "peak_source": f"{props.multi_processor_count} SMs x 32 lanes x {clk:.0f} MHz", **common,
+                    "hbm_equivalent_gbs": hbm_gbs,
+                    "note": "the codes stay in L2, so HBM bandwidth does not bound this workload; the HBM-equivalent "
+                            "rate (code bytes / kernel time) is context only"}
 
     cpu = cpu_baseline(index, q_np, nprobe, k, radius, scale, args.cpu_sample, score, model)
 
@@ -409,15 +462,8 @@ def run_cuda(args):
                 "h2d_bytes_per_step": int(qh.numel() * 4), "d2h_bytes_per_step": int(odh.numel() * 4 + oih.numel() * 4)},
         "gpu_launches": int(launches),
         "clocks": sampler.summary(),
-        "roofline": {"bound": "hbm", "kernel": scan_kernel_name(index) + " (selective LUT + list scan + top-k)",
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_source": f"of {peak_src}", "algorithmic_bytes_per_launch": int(scan_bytes),
-                     "visits_per_launch": int(visits),
-                     "traffic": SCAN_DRAM_TRAFFIC_BYTES.get(args.workload)
-                     if (args.nq is None and args.nprobe == 0 and score == 0 and metric == 0) else None},
-        "gather_roofline": {"bound": "shared-memory gathers", "achieved": gather_rate, "peak": gather_peak,
-                            "unit": "Ggather/s", "frac": gather_rate / gather_peak,
-                            "peak_source": f"{props.multi_processor_count} SMs x 32 lanes x {clk:.0f} MHz"},
+        "roofline": roofline,
+        "selection": sel_stats,
         "cpu_baseline": cpu,
     }
     if dyn_report is not None:
@@ -439,19 +485,32 @@ class _Null:
 # the CPU oracle: cpu_baseline leg and --impl reference
 # --------------------------------------------------------------------------------------------
 
+def oracle_sample_size(index, q_np, nprobe, k, radius, scale, score, want, target_s=15.0, model=None):
+    """Number of queries for one timed oracle call: `want` if given, else as many as take about
+    `target_s` seconds, estimated from a first call on 32 queries (which also pages the index in)."""
+    import oracle
+    nq = q_np.shape[0]
+    if want and want > 0:
+        return min(want, nq)
+    n0 = min(32, nq)
+    rad = radius if model is None else oracle.thresholds(index.d, index.nsub, index.dsub, q_np[:n0], model)
+    oracle.search(index, q_np[:n0], nprobe, k, radius=rad, scale=scale, score=score)
+    t0 = time.perf_counter()
+    oracle.search(index, q_np[:n0], nprobe, k, radius=rad, scale=scale, score=score)
+    rate = n0 / max(1e-6, time.perf_counter() - t0)
+    return int(max(n0, min(nq, rate * target_s)))
+
+
 def cpu_baseline(index, q_np, nprobe, k, radius, scale, sample, score=0, model=None):
     import oracle
-    sample = min(sample, q_np.shape[0])
-    if model is not None:
-        radius = oracle.thresholds(index.d, index.nsub, index.dsub, q_np[:8], model)
-    oracle.search(index, q_np[:8], nprobe, k, radius=radius, scale=scale, score=score)    # page in
+    sample = oracle_sample_size(index, q_np, nprobe, k, radius, scale, score, sample, model=model)
     t0 = time.perf_counter()
     if model is not None:
         radius = oracle.thresholds(index.d, index.nsub, index.dsub, q_np[:sample], model)
     oracle.search(index, q_np[:sample], nprobe, k, radius=radius, scale=scale, score=score)
     dt = time.perf_counter() - t0
     return {"value": sample / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"first {sample} queries of the batch, one oracle.search call, {dt:.2f} s"}
+            "sample": f"first {sample} of the batch's {q_np.shape[0]} queries, one oracle.search call, {dt:.2f} s"}
 
 
 def run_reference(args):
@@ -464,19 +523,21 @@ def run_reference(args):
                                                         metric=1 if args.metric == "ip" else 0)
     nprobe = args.nprobe or cfg.nprobes[len(cfg.nprobes) // 2]
     k = cfg.k
-    sample = min(args.cpu_sample, q_np.shape[0])
     scale = args.ref_scale
     if scale <= 0:
         # the same rule as the CUDA arm (smallest scale whose recall@100 is within 0.01 of dense),
-        # decided by the oracle on the first 1000 queries
-        ns = min(1000, q_np.shape[0])
+        # decided by the oracle on a query sample that takes it a few seconds per scale
+        ns = oracle_sample_size(index, q_np, nprobe, k, radius, 1.0, 0, 0, target_s=4.0)
+        ns = min(ns, 1000)
         _, _, (scale, _, _), sweep = pick_scale(
             lambda sc: oracle.search(index, q_np[:ns], nprobe, k, radius=radius, scale=sc)["ids"],
             lambda: oracle.search(index, q_np[:ns], nprobe, k, dense=True)["ids"], true_ids[:ns])
-        log(f"[bench] reference arm: radius scale {scale} (sweep {sweep})")
-    for _ in range(min(args.warmup, 1)):
-        oracle.search(index, q_np[:64], nprobe, k, radius=radius, scale=scale)
+        log(f"[bench] reference arm: radius scale {scale} from {ns} queries (sweep {sweep})")
     steps = min(args.steps, 5)
+    # each step: a bounded sample of the batch, sized so that all steps take about 20 s together
+    sample = oracle_sample_size(index, q_np, nprobe, k, radius, scale, 0, args.cpu_sample, target_s=20.0 / steps)
+    for _ in range(min(args.warmup, 1)):
+        oracle.search(index, q_np[:min(64, sample)], nprobe, k, radius=radius, scale=scale)
     t0 = time.perf_counter()
     for i in range(steps):
         lo = (i * sample) % max(1, q_np.shape[0] - sample + 1)
@@ -504,10 +565,13 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(CONFIGS))
+    ap.add_argument("--workload", default="c5", choices=sorted(CONFIGS),
+                    help="c5 (100 M points, 1.6 GB of codes: the one workload whose list scan streams from HBM) is "
+                         "the headline; c1-c4 fit the L2 cache")
     ap.add_argument("--nprobe", type=int, default=0)
     ap.add_argument("--nq", type=int, default=None)
-    ap.add_argument("--cpu-sample", type=int, default=10000, help="queries timed on the CPU oracle")
+    ap.add_argument("--cpu-sample", type=int, default=0,
+                    help="queries timed on the CPU oracle; 0 = as many as take about 15 s (at most the batch)")
     ap.add_argument("--ref-scale", type=float, default=0.0,
                     help="radius scale of the reference arm; 0 = chosen by the CUDA arm's recall rule")
     ap.add_argument("--dynamic-radius", action="store_true",

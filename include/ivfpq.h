@@ -264,6 +264,16 @@ int64_t ivfpq_last_launch_count(const ivfpq_index_t* index);
 int ivfpq_probe_static(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t nprobe,
                        int32_t* probe_ids, float* probe_d, void* stream);
 
+/* Status of the most recent ivfpq_probe_static call on the current device (the paper has no
+ * counterpart; it completes ivfpq_probe_static for the same callers).  That call has no workspace
+ * whose status word ivfpq_sync_status could read: its kernels record a dropped candidate or a
+ * bounded wait that ran out in the first word of the built-in array.  This reads that word back
+ * (one small copy into a host variable, then a synchronisation of `stream`; nothing is allocated)
+ * and returns IVFPQ_OK, IVFPQ_ERR_DEVICE_FLAG (the probe lists of that call are incomplete) or
+ * IVFPQ_ERR_CUDA.  Call it on the stream the probe call used, before the next probe call clears
+ * the word. */
+int ivfpq_static_status(void* stream);
+
 const char* ivfpq_error_string(int code);
 
 /* ---- test-only exports (small inputs) -------------------------------------------------------

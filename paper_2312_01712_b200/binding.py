@@ -40,7 +40,7 @@ EXPORTS = (
     "ivfpq_search_workspace_bytes", "ivfpq_search_dense", "ivfpq_search_sparse",
     "ivfpq_search_host_workspace_bytes", "ivfpq_search_host", "ivfpq_sync_status",
     "ivfpq_index_set_option", "ivfpq_last_launch_count", "ivfpq_last_stage_ms", "ivfpq_error_string",
-    "ivfpq_debug_probes", "ivfpq_debug_search", "ivfpq_probe_static", "ivfpq_query_thresholds",
+    "ivfpq_debug_probes", "ivfpq_debug_search", "ivfpq_probe_static", "ivfpq_static_status", "ivfpq_query_thresholds",
     "ivfpq_entry_stats",
 )
 
@@ -119,6 +119,8 @@ def load_library() -> ctypes.CDLL:
     lib.ivfpq_entry_stats.restype = ctypes.c_int
     lib.ivfpq_probe_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
     lib.ivfpq_probe_static.restype = ctypes.c_int
+    lib.ivfpq_static_status.argtypes = [vp]
+    lib.ivfpq_static_status.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -360,6 +362,15 @@ def ivfpq_probe_static(ix: IndexHandle, queries: torch.Tensor, nprobe: int,
     _check(load_library().ivfpq_probe_static(ix.handle, queries.data_ptr(), nq, nprobe, pid.data_ptr(),
                                              pd.data_ptr(), _stream()), "ivfpq_probe_static")
     return pid, pd
+
+
+def ivfpq_static_status() -> int:
+    """Waits for the current stream and returns IVFPQ_OK or IVFPQ_ERR_DEVICE_FLAG for the most recent
+    `ivfpq_probe_static` call on the current device (that call has no workspace to ask)."""
+    rc = load_library().ivfpq_static_status(_stream())
+    if rc not in (IVFPQ_OK, IVFPQ_ERR_DEVICE_FLAG):
+        _check(rc, "ivfpq_static_status")
+    return rc
 
 
 class ThresholdModelHandle:

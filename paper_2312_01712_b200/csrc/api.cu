@@ -331,7 +331,7 @@ static void fill_radius(SearchArgs& a, const ivfpq_radius_t* radius) {
     a.radius = radius->radius;
     a.radius_mode = radius->mode;
     a.scale = radius->scale;
-    a.miss_penalty = radius->miss_penalty;
+    a.miss_penalty = radius->miss_penalty == 0.0f ? 0.0f : radius->miss_penalty;   // -0 counts as +0
     a.score = radius->score;
 }
 

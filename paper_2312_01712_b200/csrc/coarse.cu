@@ -217,3 +217,16 @@ extern "C" int ivfpq_probe_static(const ivfpq_index_t* index, const float* queri
         return IVFPQ_ERR_CUDA;
     return IVFPQ_OK;
 }
+
+extern "C" int ivfpq_static_status(void* stream) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    unsigned char* scratch = nullptr;
+    const int rc = ivfpq::static_scratch_address(dev, &scratch);
+    if (rc != IVFPQ_OK) return rc;
+    int flags = 0;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&flags, scratch, sizeof(flags), cudaMemcpyDeviceToHost, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    return flags != 0 ? IVFPQ_ERR_DEVICE_FLAG : IVFPQ_OK;
+}

@@ -319,8 +319,11 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
     const float cmax = __uint_as_float(*cmax_bits);
     // |approx - exact| <= eps: TF32 keeps 10 mantissa bits of each factor (relative 2^-10 each, 2^-9
     // per product), summed over the dimensions by Cauchy-Schwarz and doubled by the factor -2; the
-    // second term covers fp32 accumulation and the rounding of the exact side.
-    const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + 3.8e-6f * (qn + cmax);
+    // second term covers the fp32 rounding of both sides, which grows with the number of summed
+    // terms: d accumulations in the tensor-core sum and in the squared norms, d in the exact chain
+    // (each at most 2^-24 of the running magnitude, itself at most |q|^2 + max|c|^2 up to a factor 2).
+    const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) +
+                      (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
 
     // exact squared distance by the defining arithmetic (rows are 16-byte aligned, d % 4 == 0)
     auto exact = [&](int c) {

@@ -1,7 +1,7 @@
 // Block-level streaming top-k over 64-bit keys (distance bits in the high word, id or index in
 // the low word).  Distances are non-negative fp32 (or +inf), so the unsigned order of the keys
-// is the lexicographic (distance, id) order the search returns (paper Sec. 2.1: the query "sorts
-// the results and selects the top-k"; ties by ascending id is this library's rule).
+// is the lexicographic (distance, id) order the search returns (the final ranking of all visited
+// points, paper Sec. 2.1, last paragraph; ties by ascending id is this library's rule).
 //
 // Candidates whose key is below the current threshold are appended to a shared-memory buffer.
 // When the buffer fills up, topk_select keeps the k smallest keys with a most-significant-digit

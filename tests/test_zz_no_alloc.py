@@ -38,9 +38,17 @@ def test_static_scratch_probes_equal_workspace_probes_twice(wl_small):
             out = (torch.full((nq, nprobe), -7, dtype=torch.int32, device="cuda"),
                    torch.full((nq, nprobe), -1.0, dtype=torch.float32, device="cuda"))
             ids, d = lib.ivfpq_probe_static(h, qs, nprobe, out=out)
-            torch.cuda.synchronize()
+            # the call has no workspace whose status word could be read: its own status entry point
+            assert lib.ivfpq_static_status() == lib.IVFPQ_OK
             assert torch.equal(ids, ref_ids)
             assert torch.equal(d.view(torch.int32), ref_d.view(torch.int32))
+            # with the outputs supplied, further calls leave the device's free memory where it was
+            free0 = torch.cuda.mem_get_info()[0]
+            for _ in range(3):
+                lib.ivfpq_probe_static(h, qs, nprobe, out=out)
+                assert lib.ivfpq_static_status() == lib.IVFPQ_OK
+            assert torch.cuda.mem_get_info()[0] == free0
+            assert torch.equal(out[0], ref_ids)
     finally:
         lib.ivfpq_index_free(h)
 
