@@ -291,6 +291,13 @@ def run_cuda(args):
     k = cfg.k
     nq = q_np.shape[0]
     h = lib.ivfpq_index_load(index, dev)
+    has_map = (index.nsub, index.dsub) == (16, 8) and metric == 0
+    if args.sparse_scan != "auto":
+        if args.sparse_scan == "map" and not has_map:
+            raise SystemExit("--sparse-scan map: this index shape has no entry->points map")
+        lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_SPARSE_SCAN,
+                                   lib.IVFPQ_SPARSE_SCAN_MAP if args.sparse_scan == "map" else lib.IVFPQ_SPARSE_SCAN_STREAM)
+    map_scan = has_map and args.sparse_scan == "map"
     qd = torch.from_numpy(q_np).to(dev)
     model = mh = None
     if dynamic:
@@ -420,7 +427,7 @@ def run_cuda(args):
     l2_bytes = int(getattr(props, "L2_cache_size", 126 << 20))
     hbm_gbs = scan_bytes / (scan_ms * 1e-3) / 1e9
     gather_peak = props.multi_processor_count * 32 * clk * 1e6 / 1e9            # G gathers/s
-    kernel = scan_kernel_name(index) + " (selective LUT + list scan + top-k)"
+    kernel = ("scan16x8_map_kernel" if map_scan else scan_kernel_name(index)) + " (selective LUT + list scan + top-k)"
     default_run = args.nq is None and args.nprobe == 0 and score == 0 and metric == 0 and not dynamic
     traffic = SCAN_DRAM_TRAFFIC.get(args.workload) if default_run else None
     common = {"kernel": kernel, "algorithmic_bytes_per_launch": int(scan_bytes), "visits_per_launch": int(visits),
@@ -578,6 +585,9 @@ def main():
                     help="query-specific thresholds from density maps + polynomial regressor (workload c3)")
     ap.add_argument("--metric", default="l2", choices=["l2", "ip"],
                     help="similarity of the index (l2 = the headline path)")
+    ap.add_argument("--sparse-scan", default="auto", choices=["auto", "stream", "map"],
+                    help="list scan of the sparse search on the 16x8 shape: walk the entry->points map, stream the "
+                         "codes, or let the library choose (it streams)")
     ap.add_argument("--score", default="distance", choices=sorted(SCORE_NAMES),
                     help="what the sparse search ranks by (distance = the headline path)")
     args = ap.parse_args()

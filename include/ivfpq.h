@@ -90,7 +90,9 @@ typedef struct {
 } ivfpq_index_desc_t;
 
 /* Bytes of caller-owned device memory that ivfpq_index_load needs for derived tables (codes
- * re-laid-out in 32-point interleaved blocks, list tables).  0 on invalid descriptions. */
+ * re-laid-out in 32-point interleaved blocks, list tables; for the 16 x 8 shape under L2 also the
+ * inverted index from codebook entries to points of Algorithm 1, 2 bytes per code byte plus
+ * 16 KB per 8192 points of a list).  0 on invalid descriptions. */
 size_t ivfpq_index_derived_bytes(const ivfpq_index_desc_t* desc);
 
 /* Validates the description, builds the derived tables in `derived_dev` (256-byte aligned, at
@@ -225,6 +227,31 @@ int ivfpq_sync_status(const ivfpq_index_t* index, void* workspace, void* stream)
  *   LUT+scan(+merge) stage of every search (the events are created once, on the first timed
  *   call); 0 = off (default).  Read them with ivfpq_last_stage_ms. */
 #define IVFPQ_OPT_TIMING 2
+/*   IVFPQ_OPT_SPARSE_SCAN: which list scan serves ivfpq_search_sparse on an index of 16 subspaces x
+ *   8 dimensions under L2, the shape for which ivfpq_index_load also builds the inverted index from
+ *   codebook entries to points (Algorithm 1's Map).  IVFPQ_SPARSE_SCAN_STREAM streams the codes of
+ *   every probed list as the dense search does (an unselected entry's table slot holds the
+ *   constant).  IVFPQ_SPARSE_SCAN_MAP walks the map: for every selected entry the points encoded
+ *   with it receive its table value; the other points are assigned the constant without any
+ *   look-up (Sec. 5.3, paragraph after Algorithm 2), so the scatter work follows the number of
+ *   selected entries.  IVFPQ_SPARSE_SCAN_AUTO (default) = STREAM: on B200 a table look-up costs
+ *   three instructions, while the map walk pays two shared-memory atomics per (point, selected
+ *   entry) pair and still has to visit every point's accumulator once; it was slower at every
+ *   radius measured.  Same results either way (the sums over subspaces are taken in different
+ *   orders: equal within rounding).  Other shapes have no map: MAP is refused with
+ *   IVFPQ_ERR_UNSUPPORTED. */
+#define IVFPQ_OPT_SPARSE_SCAN 3
+#define IVFPQ_SPARSE_SCAN_AUTO 0
+#define IVFPQ_SPARSE_SCAN_STREAM 1
+#define IVFPQ_SPARSE_SCAN_MAP 2
+/*   IVFPQ_OPT_TEST_FAULT (test-only): 1 = in every following search the tensor-core filtering kernel
+ *   leaves out the last centroid tile of its first CTA and shortens its wait limits to about a
+ *   millisecond, so that the bounded wait for that tile runs out.  Nothing faults and nothing is left
+ *   in flight: the kernel raises its status flag, releases its tensor memory and returns; the search
+ *   completes with unreliable probe lists and ivfpq_sync_status reports IVFPQ_ERR_DEVICE_FLAG.  Back
+ *   to 0, the next search is normal.  IVFPQ_ERR_UNSUPPORTED for indexes that the tensor-core filtering
+ *   does not serve. */
+#define IVFPQ_OPT_TEST_FAULT 4
 int ivfpq_index_set_option(ivfpq_index_t* index, int32_t option, int64_t value);
 
 /* Waits for the most recent timed search on this handle to finish and writes the device time

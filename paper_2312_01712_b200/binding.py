@@ -29,6 +29,11 @@ IVFPQ_STATIC_SCRATCH_BYTES = 8 << 20
 IVFPQ_STATIC_MAX_NLIST = 16384
 IVFPQ_OPT_NSPLIT = 1
 IVFPQ_OPT_TIMING = 2
+IVFPQ_OPT_SPARSE_SCAN = 3
+IVFPQ_OPT_TEST_FAULT = 4
+IVFPQ_SPARSE_SCAN_AUTO = 0
+IVFPQ_SPARSE_SCAN_STREAM = 1
+IVFPQ_SPARSE_SCAN_MAP = 2
 IVFPQ_METRIC_L2 = 0
 IVFPQ_METRIC_IP = 1
 IVFPQ_SCORE_DISTANCE = 0

@@ -14,7 +14,9 @@ namespace {
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 struct DerivedLayout {
-    size_t list_off_off, list_blk_off, codes_off, cbt_off, cnorm_off, total;
+    size_t list_off_off, list_blk_off, codes_off, cbt_off, cnorm_off, chunk_first_off, map_off_off, map_pos_off, total;
+    int32_t map;
+    int64_t nchunks;
     int32_t mma;
     int64_t nblocks, max_len;
     int32_t nw, vec16;
@@ -32,11 +34,12 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     if (d->ntotal > 0x7FFFFFFFll) return IVFPQ_ERR_UNSUPPORTED;  // ids are int32
     if (!d->list_offsets) return IVFPQ_ERR_INVALID_ARGUMENT;
     if (d->list_offsets[0] != 0 || d->list_offsets[d->nlist] != d->ntotal) return IVFPQ_ERR_INVALID_ARGUMENT;
-    int64_t nblocks = 0, max_len = 0;
+    int64_t nblocks = 0, max_len = 0, nchunks = 0;
     for (int c = 0; c < d->nlist; ++c) {
         const int64_t len = d->list_offsets[c + 1] - d->list_offsets[c];
         if (len < 0) return IVFPQ_ERR_INVALID_ARGUMENT;
         nblocks += (len + kPointsPerBlock - 1) / kPointsPerBlock;
+        nchunks += (len + kMapChunk - 1) / kMapChunk;
         if (len > max_len) max_len = len;
     }
     out->nw = (d->nsub + 3) / 4;
@@ -58,6 +61,18 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     out->cnorm_off = off;
     out->mma = (d->metric == IVFPQ_METRIC_L2 && coarse_mma_supported(d->d, d->nlist)) ? 1 : 0;
     if (out->mma) off = align_up(off + coarse_mma_derived_bytes(d->nlist), 256);
+    // entry -> points map of the sparsity-aware scan: the 16 x 8 shape under L2 (element indices are 32-bit)
+    out->map = (out->rot && d->nsub == 16 && d->dsub == 8 && d->ntotal > 0 && d->ntotal * 16 < ((int64_t)1 << 32)) ? 1 : 0;
+    out->nchunks = nchunks;
+    out->chunk_first_off = out->map_off_off = out->map_pos_off = off;
+    if (out->map) {
+        out->chunk_first_off = off;
+        off = align_up(off + sizeof(int32_t) * (size_t)(d->nlist + 1), 256);
+        out->map_off_off = off;
+        off = align_up(off + (size_t)nchunks * d->nsub * 256 * 4, 256);
+        out->map_pos_off = off;
+        off = align_up(off + (size_t)d->ntotal * d->nsub * 2, 256);
+    }
     out->total = off > 0 ? off : 256;
     return IVFPQ_OK;
 }
@@ -230,6 +245,17 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->cbt = reinterpret_cast<const float*>(base + dl.cbt_off);
     ix->cnorm = dl.mma ? reinterpret_cast<const float*>(base + dl.cnorm_off) : nullptr;
     ix->max_list_len = dl.max_len;
+    ix->chunk_first = dl.map ? reinterpret_cast<const int32_t*>(base + dl.chunk_first_off) : nullptr;
+    ix->map_off = dl.map ? reinterpret_cast<const uint32_t*>(base + dl.map_off_off) : nullptr;
+    ix->map_pos = dl.map ? reinterpret_cast<const uint16_t*>(base + dl.map_pos_off) : nullptr;
+    ix->nchunks = dl.nchunks;
+    {
+        // lanes per selected entry in the scatter: about the mean number of points behind one entry
+        const int64_t seg = dl.nchunks > 0 ? desc->ntotal / dl.nchunks / 256 : 0;
+        ix->map_group = seg < 6 ? 4 : (seg < 12 ? 8 : (seg < 24 ? 16 : 32));
+    }
+    ix->sparse_scan = 0;
+    ix->test_fault = 0;
     ix->device = dev;
     ix->sm_count = sms;
     ix->nsplit_opt = 0;
@@ -242,23 +268,32 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     // list tables: built on the host, copied synchronously (pageable source)
     const size_t n1 = (size_t)desc->nlist + 1;
     int64_t* blk = new (std::nothrow) int64_t[n1];
-    if (!blk) {
+    int32_t* chf = new (std::nothrow) int32_t[n1];
+    if (!blk || !chf) {
+        delete[] blk;
+        delete[] chf;
         delete ix;
         return IVFPQ_ERR_INVALID_ARGUMENT;
     }
     blk[0] = 0;
+    chf[0] = 0;
     for (int c = 0; c < desc->nlist; ++c) {
         const int64_t len = desc->list_offsets[c + 1] - desc->list_offsets[c];
         blk[c + 1] = blk[c] + (len + kPointsPerBlock - 1) / kPointsPerBlock;
+        chf[c + 1] = chf[c] + (int32_t)((len + kMapChunk - 1) / kMapChunk);
     }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemcpyAsync(base + dl.list_off_off, desc->list_offsets, n1 * 8, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(base + dl.list_blk_off, blk, n1 * 8, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && dl.map)
+        e = cudaMemcpyAsync(base + dl.chunk_first_off, chf, n1 * 4, cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);  // the host arrays may go away after return
     delete[] blk;
+    delete[] chf;
     if (e == cudaSuccess)
         e = launch_relayout(ix, desc->codes, reinterpret_cast<uint32_t*>(base + dl.codes_off),
                             reinterpret_cast<float*>(base + dl.cbt_off), st);
+    if (e == cudaSuccess) e = launch_entry_map(ix, desc->codes, st);
     if (e == cudaSuccess && ix->cnorm)
         e = launch_cnorm(ix->cent, ix->nlist, ix->d, reinterpret_cast<float*>(base + dl.cnorm_off), st);
     if (e != cudaSuccess) {
@@ -464,6 +499,16 @@ int ivfpq_index_set_option(ivfpq_index_t* index, int32_t option, int64_t value) 
         case IVFPQ_OPT_NSPLIT:
             if (value < 0 || value > 64) return IVFPQ_ERR_INVALID_ARGUMENT;
             index->nsplit_opt = (int32_t)value;
+            return IVFPQ_OK;
+        case IVFPQ_OPT_SPARSE_SCAN:
+            if (value < IVFPQ_SPARSE_SCAN_AUTO || value > IVFPQ_SPARSE_SCAN_MAP) return IVFPQ_ERR_INVALID_ARGUMENT;
+            if (value == IVFPQ_SPARSE_SCAN_MAP && !index->map_pos) return IVFPQ_ERR_UNSUPPORTED;
+            index->sparse_scan = (int32_t)value;
+            return IVFPQ_OK;
+        case IVFPQ_OPT_TEST_FAULT:
+            if (value != 0 && value != 1) return IVFPQ_ERR_INVALID_ARGUMENT;
+            if (value == 1 && !index->cnorm) return IVFPQ_ERR_UNSUPPORTED;   // the tensor-core filtering kernel is the one with bounded waits
+            index->test_fault = (int32_t)value;
             return IVFPQ_OK;
         case IVFPQ_OPT_TIMING:
             if (value != 0 && value != 1) return IVFPQ_ERR_INVALID_ARGUMENT;

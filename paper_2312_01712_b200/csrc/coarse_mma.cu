@@ -36,7 +36,8 @@ constexpr int kStages = 4;           // centroid tiles in flight
 constexpr int kMaxKBlocks = 8;       // dimension <= 256
 constexpr int kMmaThreads = 192;     // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
 constexpr int kTmemCols = 256;       // two accumulators of 128 columns
-constexpr unsigned kSpinLimit = 1u << 22;
+constexpr unsigned kSpinLimit = 1u << 22;       // polls of one bounded wait
+constexpr unsigned kSpinLimitTest = 1u << 16;   // ... while the test-only fault option is on (about a millisecond)
 constexpr int kCandCap = kTopkCap;   // centroids that may pass the cut before the exact fallback
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
@@ -61,8 +62,9 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: false (and the abort word set) when it ran out or somebody else gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int* status) {
-    for (unsigned i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_word, int* status,
+                                          unsigned limit) {
+    for (unsigned i = 0; i < limit; ++i) {
         if (mbar_try(bar, parity)) return true;
         if (*abort_word) return false;
     }
@@ -134,7 +136,11 @@ struct MmaShared {
 __global__ void __launch_bounds__(kMmaThreads, 1)
 coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c,
                   const float* __restrict__ cnorm, int nqc, int nlist, int kblocks, float* __restrict__ out,
-                  int* __restrict__ status) {
+                  int* __restrict__ status, int skip_last_load) {
+    // Test-only: with skip_last_load the producer of the first CTA leaves out its very last centroid tile
+    // (nothing is handed to the copy engine, nothing is left in flight), so the wait for that tile runs
+    // out: the way the bounded waits give up is then observable without any fault.
+    const unsigned limit = skip_last_load ? kSpinLimitTest : kSpinLimit;
     extern __shared__ __align__(1024) unsigned char dyn[];
     // the swizzled tiles need 1024-byte alignment in the shared window
     const uint32_t dyn_addr = smem_u32(dyn);
@@ -182,8 +188,9 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y) {
                 for (int kb = 0; kb < kblocks && ok; ++kb, ++it) {
                     const unsigned s = it % kStages;
-                    ok = mbar_wait(smem_u32(&sh->empty[s]), ((it / kStages) & 1) ^ 1, abort_word, status);
+                    ok = mbar_wait(smem_u32(&sh->empty[s]), ((it / kStages) & 1) ^ 1, abort_word, status, limit);
                     if (!ok) break;
+                    if (skip_last_load && blockIdx.x == 0 && blockIdx.y == 0 && ct + (int)gridDim.y >= ntile && kb == kblocks - 1) break;
                     mbar_expect_tx(smem_u32(&sh->full[s]), kTileBytes);
                     tma_load_2d(b_smem + s * kTileBytes, &map_c, kb * kKBlock, ct * kTileN, smem_u32(&sh->full[s]));
                 }
@@ -192,16 +199,16 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     } else if (warp == 1) {
         if (lane == 0) {
             // ---- MMA issuer ----
-            bool ok = mbar_wait(smem_u32(&sh->q_full), 0, abort_word, status);
+            bool ok = mbar_wait(smem_u32(&sh->q_full), 0, abort_word, status, limit);
             unsigned it = 0, t = 0;
             for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y, ++t) {
                 const unsigned buf = t & 1;
-                ok = mbar_wait(smem_u32(&sh->acc_empty[buf]), ((t >> 1) & 1) ^ 1, abort_word, status);
+                ok = mbar_wait(smem_u32(&sh->acc_empty[buf]), ((t >> 1) & 1) ^ 1, abort_word, status, limit);
                 if (!ok) break;
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks && ok; ++kb, ++it) {
                     const unsigned s = it % kStages;
-                    ok = mbar_wait(smem_u32(&sh->full[s]), (it / kStages) & 1, abort_word, status);
+                    ok = mbar_wait(smem_u32(&sh->full[s]), (it / kStages) & 1, abort_word, status, limit);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
@@ -222,7 +229,7 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         bool ok = true;
         for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y, ++t) {
             const unsigned buf = t & 1;
-            ok = mbar_wait(smem_u32(&sh->acc_full[buf]), (t >> 1) & 1, abort_word, status);
+            ok = mbar_wait(smem_u32(&sh->acc_full[buf]), (t >> 1) & 1, abort_word, status, limit);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll 1
@@ -476,7 +483,8 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
     if (e != cudaSuccess) return e;
     const float* cnorm = ix->cnorm;
     const unsigned* cmax = reinterpret_cast<const unsigned*>(reinterpret_cast<const char*>(cnorm) + align_up((size_t)ix->nlist * 4, 256));
-    coarse_mma_kernel<<<dim3(qtiles, csplit), kMmaThreads, smem, st>>>(map_q, map_c, cnorm, nqc, ix->nlist, kblocks, tile, status);
+    coarse_mma_kernel<<<dim3(qtiles, csplit), kMmaThreads, smem, st>>>(map_q, map_c, cnorm, nqc, ix->nlist, kblocks, tile, status,
+                                                                       ix->test_fault);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const size_t smem2 = (size_t)kTopkCap * 8 + (size_t)kCandCap * 4 + align_up((size_t)ix->d * 4, 16);

@@ -11,12 +11,14 @@ namespace ivfpq {
 constexpr int kPointsPerBlock = 32;  // points per interleaved code block (one warp, one point per lane)
 constexpr int kScanThreads = 256;    // threads per scan CTA (= max entries per codebook)
 constexpr int kTopkCap = 2048;       // candidate buffer slots per CTA (>= IVFPQ_MAX_K + kScanThreads)
+constexpr int kMapChunk = 8192;      // points per chunk of the entry -> points map (entry_map.cu)
 
 // Device status bits (workspace status word).
 constexpr int kFlagBadList = 1;   // a probed cluster id or code block was out of range and was skipped
 constexpr int kFlagOverflow = 2;  // the candidate buffer would have overflowed; the candidate was dropped
 constexpr int kFlagTimeout = 4;   // a bounded wait between cooperating warps ran out
 constexpr int kFlagLayout = 8;    // the kernel's shared-memory layout does not fit the window offset it was given
+constexpr int kFlagMap = 16;      // the entry -> points map disagrees with the codes (stage-dump instances check this)
 
 inline __host__ __device__ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -45,6 +47,14 @@ struct ivfpq_index {
     int32_t block_bytes;      // bytes of one 32-point code block in the rotated layout
     const float* cbt;         // [group][entry 0..255][column][dsub]
     const float* cnorm;       // [nlist] squared centroid norms + their maximum (tensor-core filtering), or null
+    // entry -> points map (entry_map.cu; 16 x 8 shape under L2 only, null otherwise)
+    const int32_t* chunk_first;  // [nlist+1] chunks before each list
+    const uint32_t* map_off;     // [nchunks][nsub][256]: first position | point count << 16 of every entry
+    const uint16_t* map_pos;     // [ntotal * nsub]
+    int64_t nchunks;
+    int32_t map_group;        // lanes that share one entry's point list in the scatter (4, 8, 16 or 32)
+    int32_t sparse_scan;      // IVFPQ_OPT_SPARSE_SCAN
+    int32_t test_fault;       // IVFPQ_OPT_TEST_FAULT
     int64_t max_list_len;
     // host state
     int32_t device;
@@ -115,6 +125,7 @@ bool rot_supported(int nsub, int dsub);
 // Tensor-core filtering (coarse_mma.cu).
 bool coarse_mma_supported(int d, int nlist);
 size_t coarse_mma_derived_bytes(int nlist);
+cudaError_t launch_entry_map(const ivfpq_index* ix, const uint8_t* codes, cudaStream_t st);
 cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st);
 cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe,
                               float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,

@@ -13,6 +13,8 @@
 //      one table value per subspace (step D);
 //   4. feeds (distance, id) into a CTA-wide streaming top-k.
 // The table is never written to global memory.
+#include <math.h>
+
 #include "common.cuh"
 #include "scan_common.cuh"
 #include "topk.cuh"
@@ -465,6 +467,14 @@ cudaError_t dispatch(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, 
 
 }  // namespace
 
+// Which list scan serves a sparsity-aware search of the 16 x 8 shape: the code stream (work
+// proportional to the list lengths) unless the caller asked for the walk through the entry ->
+// points map (work proportional to the selected entries; measured slower on this hardware at every
+// radius tried, see the option's description).
+static bool use_entry_map(const ivfpq_index* ix, const SearchArgs& a) {
+    return !a.dense && ix->map_pos && ix->sparse_scan == IVFPQ_SPARSE_SCAN_MAP;
+}
+
 cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws, cudaStream_t st,
                         int64_t* launches) {
     const ivfpq_index* ix = a.ix;
@@ -476,6 +486,10 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     sp.codes_il = ix->codes_il;
     sp.list_off = ix->list_off;
     sp.list_blk = ix->list_blk;
+    sp.chunk_first = ix->chunk_first;
+    sp.map_off = ix->map_off;
+    sp.map_pos = ix->map_pos;
+    sp.map_group = ix->map_group;
     sp.d = ix->d;
     sp.nlist = ix->nlist;
     sp.nsub = ix->nsub;
@@ -512,6 +526,8 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     const bool ip = ix->metric == IVFPQ_METRIC_IP;
     if (ip)
         e = a.debug ? launch_ip<true>(sp, grid, smem, st) : launch_ip<false>(sp, grid, smem, st);
+    else if (pers_shape(ix) && use_entry_map(ix, a))
+        e = launch_scan16x8_map(ix, sp, grid, a.debug, a.nprobe, st);
     else if (pers_shape(ix))
         e = launch_scan16x8(ix, sp, grid, a.debug, a.nprobe, st);
     else if (ix->rot)

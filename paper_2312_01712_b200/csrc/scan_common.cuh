@@ -13,6 +13,10 @@ struct ScanParams {
     const uint32_t* codes_il;
     const int64_t* list_off;
     const int64_t* list_blk;
+    const int32_t* chunk_first;   // entry -> points map (entry_map.cu), null when the index has none
+    const uint32_t* map_off;
+    const uint16_t* map_pos;
+    int map_group;
     int d, nlist, nsub, dsub, ksub, nw;
     int vec16;   // generic layout: 1 = code words grouped by four (16-byte lane loads)
     const float* queries;
@@ -61,6 +65,10 @@ __device__ __forceinline__ float table_value(int score, bool hit, float d2, floa
 // specialised instance.
 cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, bool debug,
                             int nprobe, cudaStream_t st);
+
+// Sparsity-aware scan of the 16 x 8 quantizer through the entry -> points map (scan16x8_map.cu).
+cudaError_t launch_scan16x8_map(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
+                                 cudaStream_t st);
 
 // Persistent scan for the 16 x 8 quantizer, 16 or 32 warps per SM (scan16x8.cu).
 cudaError_t launch_scan16x8(const ivfpq_index* ix, const ScanParams& sp, int64_t nitems, bool debug, int nprobe,
