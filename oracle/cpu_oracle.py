@@ -75,6 +75,8 @@ def _lib() -> ctypes.CDLL:
         lib.oracle_search_ip.restype = i32
         lib.oracle_thresholds.argtypes = [i32, i32, i32, vp, i64, i32, i32, vp, vp, vp, vp, vp]
         lib.oracle_thresholds.restype = i32
+        lib.oracle_thresholds_knn.argtypes = [i32, i32, i32, i32, i32, vp, vp, vp, i64, i32, i32, vp, vp]
+        lib.oracle_thresholds_knn.restype = i32
         lib.oracle_num_threads.restype = i32
         lib.oracle_set_num_threads.argtypes = [i32]
         _LIB = lib
@@ -198,6 +200,24 @@ def thresholds(d: int, nsub: int, dsub: int, queries: np.ndarray, model) -> np.n
                                   _p(dens), _p(org), _p(inv), _p(cf), _p(out))
     if rc != 0:
         raise ValueError(f"oracle_thresholds failed: {rc}")
+    return out
+
+
+def thresholds_knn(index, queries: np.ndarray, kth: int, coef: np.ndarray) -> np.ndarray:
+    """Dynamic thresholds [nq, nsub] fp32 for subspaces of any width: a per-subspace polynomial
+    (`coef` [nsub, degree + 1], ascending powers) of the distance from the query's residual
+    projection (against its nearest cluster) to its `kth`-nearest codebook entry."""
+    q = _c(queries, np.float32)
+    cent = _c(index.coarse_centroids, np.float32)
+    cb = _c(index.codebooks, np.float32)
+    cf = _c(coef, np.float32)
+    if cf.ndim != 2 or cf.shape[0] != index.nsub:
+        raise ValueError("coef must be [nsub, degree + 1]")
+    out = np.empty((q.shape[0], index.nsub), np.float32)
+    rc = _lib().oracle_thresholds_knn(index.d, index.nlist, index.nsub, index.dsub, index.ksub, _p(cent), _p(cb),
+                                      _p(q), q.shape[0], int(kth), cf.shape[1] - 1, _p(cf), _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle_thresholds_knn failed: {rc}")
     return out
 
 

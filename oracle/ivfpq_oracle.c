@@ -333,6 +333,65 @@ int oracle_thresholds(int d, int nsub, int dsub, const float* queries, int64_t n
     return 0;
 }
 
+static int float_less(const void* a, const void* b) {
+    const float x = *(const float*)a, y = *(const float*)b;
+    return x < y ? -1 : (x > y ? 1 : 0);
+}
+
+/*
+ * Dynamic thresholds for subspaces of any width (stand-in for the density map of Sec. 4.1
+ * "Determining Proper Threshold", which is a 2-d grid and exists for 2-d subspaces only).  The local
+ * density around a query's projection is measured by how close its kth-nearest codebook entry is:
+ * the codebook is a k-means quantizer of the residual projections, so its entries crowd where the
+ * data does.  As in the paper, a per-subspace regression polynomial turns the measurement into the
+ * threshold; with the coefficients (0, 1) the threshold is the kth-nearest-entry distance itself.
+ *   projection  the residual against the query's nearest cluster (filtering with one probe, ties
+ *               to the smaller cluster id): the frame the codebooks were trained in
+ *   measurement v = sqrtf(kth smallest over the ksub entries e of |r_s - e|^2), the squared
+ *               distances by the table arithmetic of S2 (fmaf chain, ascending dimension)
+ *   radius[q][s] = max(0, polynomial_s(v)), Horner evaluation with fmaf from the highest power
+ *   coef [nsub][degree+1], ascending powers; 1 <= kth <= ksub
+ */
+int oracle_thresholds_knn(int d, int nlist, int nsub, int dsub, int ksub, const float* cent, const float* codebooks,
+                          const float* queries, int64_t nq, int kth, int degree, const float* coef, float* radius) {
+    if (d != nsub * dsub || nlist <= 0 || ksub <= 0 || ksub > 256 || kth < 1 || kth > ksub || degree < 0) return -2;
+    for (int64_t qi = 0; qi < nq; ++qi) {
+        const float* q = queries + qi * d;
+        int best = 0;
+        float bestd = 0.0f;
+        for (int c = 0; c < nlist; ++c) {
+            float a = 0.0f;
+            for (int j = 0; j < d; ++j) {
+                const float t = q[j] - cent[(size_t)c * d + j];
+                a = fmaf(t, t, a);
+            }
+            if (c == 0 || a < bestd) {
+                bestd = a;
+                best = c;
+            }
+        }
+        for (int s = 0; s < nsub; ++s) {
+            float d2[256];
+            for (int e = 0; e < ksub; ++e) {
+                float a = 0.0f;
+                for (int j = 0; j < dsub; ++j) {
+                    const float r = q[s * dsub + j] - cent[(size_t)best * d + s * dsub + j];
+                    const float t = r - codebooks[((size_t)s * ksub + e) * dsub + j];
+                    a = fmaf(t, t, a);
+                }
+                d2[e] = a;
+            }
+            qsort(d2, (size_t)ksub, sizeof(float), float_less);
+            const float v = sqrtf(d2[kth - 1]);
+            const float* cf = coef + (size_t)s * (degree + 1);
+            float acc = cf[degree];
+            for (int i = degree - 1; i >= 0; --i) acc = fmaf(acc, v, cf[i]);
+            radius[qi * nsub + s] = acc > 0.0f ? acc : 0.0f;
+        }
+    }
+    return 0;
+}
+
 /*
  * Entry usage and locality statistics of the neighbours of a query (Sec. 3.2 "Sparsity of Codebook
  * Entries Used by Top-k Neighbors" and Sec. 3.3 "Spatial Locality of Codebook Entries Used by Top-k
