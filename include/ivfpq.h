@@ -160,6 +160,25 @@ typedef struct {
 int ivfpq_query_thresholds(const ivfpq_index_t* index, const float* queries, int64_t nq,
                            const ivfpq_threshold_model_t* model, float* radius_out, void* stream);
 
+/* Query-specific thresholds for subspaces of any width.  The density map above is a 2-d grid; for
+ * wider subspaces the local density around the query's projection is measured by how close its
+ * kth-nearest codebook entry is (the codebook is a k-means quantizer of the residual projections,
+ * so its entries crowd where the data does), and, as in Sec. 4.1, a per-subspace regression
+ * polynomial turns the measurement into the threshold:
+ *   radius_out[q][s] = max(0, polynomial_s(v)),  v = sqrt(kth smallest over the entries e of
+ *   |r_s - e|^2),  r = query - its nearest cluster centroid (ties to the smaller cluster id).
+ * Squared distances by the table arithmetic (fused multiply-add chain over ascending dimensions),
+ * correctly rounded square root, Horner evaluation from the highest power with one fused
+ * multiply-add per coefficient.  coef dev [nsub][degree + 1], ascending powers; with (0, 1) the
+ * threshold is the kth-nearest-entry distance itself (the mean of its square over queries is what the
+ * static radius calibration uses).  1 <= kth <= ksub, 0 <= degree <= 8, nq <= 2^24, L2 indexes:
+ * IVFPQ_ERR_UNSUPPORTED otherwise.  The nearest clusters come from the filtering stage with one
+ * probe, which needs `workspace` of ivfpq_search_workspace_bytes(index, nq, 1, 1); queries as for
+ * the search calls.  Asynchronous on `stream`; allocates nothing. */
+int ivfpq_query_thresholds_knn(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t kth,
+                               int32_t degree, const float* coef, float* radius_out, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
 /* Entry usage and locality statistics of each query's neighbours (Sec. 3.2 "Sparsity of Codebook
  * Entries Used by Top-k Neighbors", Sec. 3.3 "Spatial Locality of Codebook Entries Used by Top-k
  * Neighbors"); an analysis tool for choosing radii, not a step of the search.

@@ -46,6 +46,7 @@ EXPORTS = (
     "ivfpq_search_host_workspace_bytes", "ivfpq_search_host", "ivfpq_sync_status",
     "ivfpq_index_set_option", "ivfpq_last_launch_count", "ivfpq_last_stage_ms", "ivfpq_error_string",
     "ivfpq_debug_probes", "ivfpq_debug_search", "ivfpq_probe_static", "ivfpq_static_status", "ivfpq_query_thresholds",
+    "ivfpq_query_thresholds_knn",
     "ivfpq_entry_stats",
 )
 
@@ -120,6 +121,8 @@ def load_library() -> ctypes.CDLL:
     lib.ivfpq_debug_search.restype = ctypes.c_int
     lib.ivfpq_query_thresholds.argtypes = [vp, vp, i64, ctypes.POINTER(ivfpq_threshold_model_t), vp, vp]
     lib.ivfpq_query_thresholds.restype = ctypes.c_int
+    lib.ivfpq_query_thresholds_knn.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.ivfpq_query_thresholds_knn.restype = ctypes.c_int
     lib.ivfpq_entry_stats.argtypes = [vp, vp, vp, i64, vp, i32, vp, vp, vp, vp]
     lib.ivfpq_entry_stats.restype = ctypes.c_int
     lib.ivfpq_probe_static.argtypes = [vp, vp, i64, i32, vp, vp, vp]
@@ -376,6 +379,27 @@ def ivfpq_static_status() -> int:
     if rc not in (IVFPQ_OK, IVFPQ_ERR_DEVICE_FLAG):
         _check(rc, "ivfpq_static_status")
     return rc
+
+
+def ivfpq_query_thresholds_knn(ix: IndexHandle, queries: torch.Tensor, kth: int, coef: torch.Tensor,
+                               out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Query-specific thresholds [nq, nsub] from the distance to the kth-nearest codebook entry
+    (`coef` [nsub, degree + 1] fp32 on the device, ascending powers)."""
+    if queries.dtype != torch.float32 or not queries.is_cuda or not queries.is_contiguous() or queries.dim() != 2 \
+            or queries.shape[1] != ix.d:
+        raise ValueError("queries must be a contiguous fp32 CUDA tensor [nq, d]")
+    if coef.dtype != torch.float32 or not coef.is_cuda or not coef.is_contiguous() or coef.dim() != 2 \
+            or coef.shape[0] != ix.nsub:
+        raise ValueError("coef must be a contiguous fp32 CUDA tensor [nsub, degree + 1]")
+    nq = queries.shape[0]
+    lib = load_library()
+    ws = ix.workspace(int(lib.ivfpq_search_workspace_bytes(ix.handle, nq, 1, 1)))
+    if out is None:
+        out = torch.empty((nq, ix.nsub), dtype=torch.float32, device=queries.device)
+    _check(lib.ivfpq_query_thresholds_knn(ix.handle, queries.data_ptr(), nq, int(kth), coef.shape[1] - 1, coef.data_ptr(),
+                                          out.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "ivfpq_query_thresholds_knn")
+    return out
 
 
 class ThresholdModelHandle:

@@ -329,6 +329,31 @@ int ivfpq_query_thresholds(const ivfpq_index_t* index, const float* queries, int
     return IVFPQ_OK;
 }
 
+int ivfpq_query_thresholds_knn(const ivfpq_index_t* index, const float* queries, int64_t nq, int32_t kth, int32_t degree,
+                               const float* coef, float* radius_out, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+    if (!index || !queries || !coef || !radius_out || !workspace || nq <= 0) return IVFPQ_ERR_INVALID_ARGUMENT;
+    if (index->metric != IVFPQ_METRIC_L2) return IVFPQ_ERR_UNSUPPORTED;
+    if (kth < 1 || kth > index->ksub || degree < 0 || degree > 8 || nq > (int64_t)1 << 24) return IVFPQ_ERR_UNSUPPORTED;
+    // the nearest cluster of every query: the filtering stage with one probe, into the workspace
+    SearchArgs a{};
+    a.ix = index;
+    a.queries = queries;
+    a.nq = nq;
+    a.nprobe = 1;
+    a.k = 1;
+    a.dense = true;
+    const int rc = run_search(a, workspace, workspace_bytes, stream, true);
+    if (rc != IVFPQ_OK) return rc;
+    const WorkspaceLayout wl = plan_workspace(index, nq, 1, 1);
+    char* ws = static_cast<char*>(workspace);
+    if (launch_thresholds_knn(index, queries, nq, reinterpret_cast<const int32_t*>(ws + wl.probe_ids_off), kth, degree, coef,
+                              radius_out, reinterpret_cast<int*>(ws + wl.status_off),
+                              reinterpret_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return IVFPQ_ERR_CUDA;
+    return IVFPQ_OK;
+}
+
 int ivfpq_entry_stats(const ivfpq_index_t* index, const uint8_t* codes, const float* queries, int64_t nq,
                       const int64_t* neighbor_pos, int32_t k, int32_t* usage_out,
                       unsigned long long* rank_hist, int32_t* flags, void* stream) {

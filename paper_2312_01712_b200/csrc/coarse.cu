@@ -137,14 +137,24 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
                           int* status, cudaStream_t st, int64_t* launches) {
     // tensor-core proposal + exact decision when the shape allows it (16-byte aligned rows)
     const bool ip = ix->metric == IVFPQ_METRIC_IP;   // the tensor-core path and its error bound are written for L2
-    const bool mma = !ip && ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
-                     (reinterpret_cast<uintptr_t>(ix->cent) & 15) == 0;
+    const bool mma_shape = !ip && ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
+                           (reinterpret_cast<uintptr_t>(ix->cent) & 15) == 0;
+    const int64_t qchunk_row = qchunk;   // queries whose full rows fit the scratch region (the plain kernels need those)
+    bool mma = mma_shape;
+    if (mma && coarse_mma_fused(ix->nlist, nprobe) && !ix->test_fault) {
+        // the fused path needs far less scratch per query than a full row: larger query chunks in the same region
+        const int64_t fit = (int64_t)(((size_t)qchunk * ix->nlist * 4 - 16) / coarse_mma_fused_bytes_per_query(ix->nlist));
+        if (fit > qchunk) qchunk = fit < nq ? fit : nq;
+    }
     for (int64_t q0 = 0; q0 < nq; q0 += qchunk) {
-        const int nqc = (int)((nq - q0 < qchunk) ? (nq - q0) : qchunk);
+        int nqc = (int)((nq - q0 < qchunk) ? (nq - q0) : qchunk);
         if (mma) {
             const cudaError_t e = launch_coarse_mma(ix, queries, q0, nqc, nprobe, coarse_tile, probe_ids, probe_d, status, st, launches);
             if (e == cudaSuccess) continue;
             if (e != cudaErrorNotSupported) return e;
+            mma = false;   // the tensor maps could not be built: the plain kernels, in chunks of full rows
+            qchunk = qchunk_row;
+            nqc = (int)((nq - q0 < qchunk) ? (nq - q0) : qchunk);
         }
         dim3 grid((ix->nlist + TC - 1) / TC, (nqc + TQ - 1) / TQ);
         if (ip) {

@@ -17,6 +17,16 @@
 //      arithmetic and the nprobe smallest (distance, cluster id) are returned.  When the cut lets
 //      too many centroids through, the CTA evaluates all of them exactly instead.
 //
+//   Many clusters, few probes (nlist >= 8192, nprobe <= 64): the [queries][nlist] tile is never
+//   written.  A first pass runs the same kernel over the first quarter of the centroids only (at
+//   most 4096; a random sample of the clusters: k-means was seeded with random points); probe_bound_kernel takes each
+//   query's nprobe-th smallest value of that sample, which is an upper bound of the nprobe-th
+//   smallest over all clusters, and adds twice the error bound; the main pass compares every
+//   accumulator value with that cut in the epilogue and appends only the survivors (value,
+//   cluster) to a short per-query list (a few times nprobe entries), from which
+//   probe_rerank_kernel proceeds as it does from a full row.  A list that overflows falls back to
+//   the exact evaluation of all clusters for that query.
+//
 // Every wait on an mbarrier is bounded; a wait that runs out raises the status flag, the roles
 // leave their loops, the tensor memory is released and the kernel returns.
 #include <cuda.h>
@@ -32,9 +42,10 @@ constexpr int kTileM = 128;          // queries per CTA tile (= TMEM lanes)
 constexpr int kTileN = 128;          // centroids per MMA tile (= TMEM columns per accumulator)
 constexpr int kKBlock = 32;          // fp32 elements per 128-byte swizzle row
 constexpr int kTileBytes = kTileM * kKBlock * 4;   // one [128 rows][128 bytes] tile: 16 KB
-constexpr int kStages = 4;           // centroid tiles in flight
+constexpr int kStages = 8;           // centroid tiles in flight, at most (as many as the shared memory holds beside the query tiles)
 constexpr int kMaxKBlocks = 8;       // dimension <= 256
-constexpr int kMmaThreads = 192;     // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int kEpiWarps = 8;         // two per tensor-memory lane quarter, 64 columns of the tile each
+constexpr int kMmaThreads = 64 + 32 * kEpiWarps;   // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
 constexpr int kTmemCols = 256;       // two accumulators of 128 columns
 constexpr unsigned kSpinLimit = 1u << 22;       // polls of one bounded wait
 constexpr unsigned kSpinLimitTest = 1u << 16;   // ... while the test-only fault option is on (about a millisecond)
@@ -129,6 +140,8 @@ struct MmaShared {
     unsigned long long acc_empty[2];
     uint32_t tmem_base;
     int abort_word;
+    float cn[2][kTileN];   // squared norms of the centroids of the tile in work and of the next one
+    int epi_stop[2];       // what the epilogue warps agree on after their barrier: somebody gave up
 };
 
 // out[(q - q0) * nlist + c] = cnorm[c] - 2 q.c (TF32 products), q in [q0, q0 + nqc), all c.
@@ -136,7 +149,11 @@ struct MmaShared {
 __global__ void __launch_bounds__(kMmaThreads, 1)
 coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c,
                   const float* __restrict__ cnorm, int nqc, int nlist, int kblocks, float* __restrict__ out,
-                  int* __restrict__ status, int skip_last_load) {
+                  int* __restrict__ status, int skip_last_load, int ntile_run, int out_stride,
+                  const float* __restrict__ cutp, int* __restrict__ ccount, uint2* __restrict__ cand, int ccap, int nstages) {
+    // ntile_run: centroid tiles to process (the first ones); out_stride: floats per row of `out`.
+    // cutp != null: nothing is written to `out`; values at or under the row's cut are appended to
+    // cand[q][ccount[q]++] (up to ccap entries are stored, the count keeps running).
     // Test-only: with skip_last_load the producer of the first CTA leaves out its very last centroid tile
     // (nothing is handed to the copy engine, nothing is left in flight), so the wait for that tile runs
     // out: the way the bounded waits give up is then observable without any fault.
@@ -148,22 +165,22 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     unsigned char* base = dyn + pad;
     const uint32_t q_smem = dyn_addr + pad;                                   // kblocks tiles
     const uint32_t b_smem = q_smem + (uint32_t)kblocks * kTileBytes;          // kStages tiles
-    MmaShared* sh = reinterpret_cast<MmaShared*>(base + (size_t)(kblocks + kStages) * kTileBytes);
+    MmaShared* sh = reinterpret_cast<MmaShared*>(base + (size_t)(kblocks + nstages) * kTileBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int qt = blockIdx.x;
-    const int ntile = (nlist + kTileN - 1) / kTileN;
+    const int ntile = ntile_run;
     volatile int* abort_word = &sh->abort_word;
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&sh->q_full), 1);
-        for (int i = 0; i < kStages; ++i) {
+        for (int i = 0; i < nstages; ++i) {
             mbar_init(smem_u32(&sh->full[i]), 1);
             mbar_init(smem_u32(&sh->empty[i]), 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&sh->acc_full[i]), 1);
-            mbar_init(smem_u32(&sh->acc_empty[i]), 4);
+            mbar_init(smem_u32(&sh->acc_empty[i]), kEpiWarps);
         }
         sh->abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -187,8 +204,8 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             bool ok = true;
             for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y) {
                 for (int kb = 0; kb < kblocks && ok; ++kb, ++it) {
-                    const unsigned s = it % kStages;
-                    ok = mbar_wait(smem_u32(&sh->empty[s]), ((it / kStages) & 1) ^ 1, abort_word, status, limit);
+                    const unsigned s = it % (unsigned)nstages;
+                    ok = mbar_wait(smem_u32(&sh->empty[s]), ((it / (unsigned)nstages) & 1) ^ 1, abort_word, status, limit);
                     if (!ok) break;
                     if (skip_last_load && blockIdx.x == 0 && blockIdx.y == 0 && ct + (int)gridDim.y >= ntile && kb == kblocks - 1) break;
                     mbar_expect_tx(smem_u32(&sh->full[s]), kTileBytes);
@@ -207,8 +224,8 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks && ok; ++kb, ++it) {
-                    const unsigned s = it % kStages;
-                    ok = mbar_wait(smem_u32(&sh->full[s]), (it / kStages) & 1, abort_word, status, limit);
+                    const unsigned s = it % (unsigned)nstages;
+                    ok = mbar_wait(smem_u32(&sh->full[s]), (it / (unsigned)nstages) & 1, abort_word, status, limit);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll
@@ -221,45 +238,112 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
         }
     } else {
-        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. + 31 = query rows of the tile ----
+        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. + 31 = query rows of the tile; the two
+        //      warps of a lane quarter take 64 columns each.  The squared norms of a tile's centroids are
+        //      staged in shared memory one tile ahead (every wait here is exposed: one warp per role). ----
         const int quarter = warp & 3;
+        const int chalf = (warp - 2) >> 2;            // 0: columns 0..63, 1: columns 64..127
+        const int et = threadIdx.x - 64;              // 0 .. 255 among the epilogue threads
         const int row = quarter * 32 + lane;
         const int q = qt * kTileM + row;
+        const float cut = (cutp != nullptr && q < nqc) ? cutp[q] : 0.0f;
+        const float kInf = __int_as_float(0x7F800000);
+        auto epi_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory"); };
+        if (et < kTileN) {
+            const int c = blockIdx.y * kTileN + et;
+            sh->cn[0][et] = (blockIdx.y < ntile && c < nlist) ? __ldg(cnorm + c) : kInf;
+        }
+        epi_sync();
+        // All epilogue warps meet at a named barrier once per tile, so they must leave the loop in the
+        // same iteration: whether somebody gave up is read by one thread before the barrier and by
+        // everybody after it (two slots: a slot is rewritten only after the following barrier).
         unsigned t = 0;
-        bool ok = true;
-        for (int ct = blockIdx.y; ct < ntile && ok; ct += gridDim.y, ++t) {
+        for (int ct = blockIdx.y; ct < ntile; ct += gridDim.y, ++t) {
             const unsigned buf = t & 1;
-            ok = mbar_wait(smem_u32(&sh->acc_full[buf]), (t >> 1) & 1, abort_word, status, limit);
-            if (!ok) break;
+            float cn_next = kInf;   // this thread's share of the next tile's norms: requested now, stored after the tile
+            if (et < kTileN && ct + (int)gridDim.y < ntile) {
+                const int c = (ct + (int)gridDim.y) * kTileN + et;
+                if (c < nlist) cn_next = __ldg(cnorm + c);
+            }
+            const bool ok = mbar_wait(smem_u32(&sh->acc_full[buf]), (t >> 1) & 1, abort_word, status, limit);
+            if (ok) {
             tc_fence_after();
-#pragma unroll 1
-            for (int cc = 0; cc < kTileN / 32; ++cc) {
+            const float* cns = sh->cn[buf];
+            // warp-collective: |c|^2 - 2 q.c of the 32 columns of group cc (+inf beyond the last centroid)
+            auto values = [&](int cc, float (&val)[32]) {
                 uint32_t v[32];
                 tc_load_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + buf * kTileN + cc * 32, v);
-                const int c0 = ct * kTileN + cc * 32;
-                if (q < nqc) {
-                    float* dst = out + (size_t)q * nlist + c0;
-                    if (c0 + 32 <= nlist && (nlist & 3) == 0) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4) {
-                            const float4 cn = __ldg(reinterpret_cast<const float4*>(cnorm + c0 + i));
-                            float4 o;
-                            o.x = fmaf(-2.0f, __uint_as_float(v[i + 0]), cn.x);
-                            o.y = fmaf(-2.0f, __uint_as_float(v[i + 1]), cn.y);
-                            o.z = fmaf(-2.0f, __uint_as_float(v[i + 2]), cn.z);
-                            o.w = fmaf(-2.0f, __uint_as_float(v[i + 3]), cn.w);
-                            *reinterpret_cast<float4*>(dst + i) = o;
+                for (int i = 0; i < 32; i += 4) {
+                    const float4 x = *reinterpret_cast<const float4*>(cns + cc * 32 + i);
+                    val[i] = fmaf(-2.0f, __uint_as_float(v[i]), x.x);
+                    val[i + 1] = fmaf(-2.0f, __uint_as_float(v[i + 1]), x.y);
+                    val[i + 2] = fmaf(-2.0f, __uint_as_float(v[i + 2]), x.z);
+                    val[i + 3] = fmaf(-2.0f, __uint_as_float(v[i + 3]), x.w);
+                }
+            };
+            if (cutp != nullptr) {
+                // Fused decision: only what may belong to the probe list leaves the kernel.  First pass
+                // over the warp's two column groups: which values are at or under the row's cut; one
+                // counter update per row and half tile (a global atomic per surviving value would be
+                // waited for one after the other); second pass over the groups that hold survivors.
+                uint32_t masks[2];
+                int total = 0;
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    float val[32];
+                    values(2 * chalf + g, val);
+                    uint32_t pass = 0;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) pass |= (val[i] <= cut ? 1u : 0u) << i;   // +inf never passes a finite cut
+                    if (q >= nqc) pass = 0;
+                    masks[g] = pass;
+                    total += __popc(pass);
+                }
+                int slot = total > 0 ? atomicAdd(ccount + q, total) : 0;
+#pragma unroll
+                for (int g = 0; g < 2; ++g) {
+                    if (__any_sync(0xFFFFFFFFu, masks[g] != 0u)) {
+                        float val[32];
+                        values(2 * chalf + g, val);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            if ((masks[g] >> i) & 1u) {
+                                if (slot < ccap)
+                                    cand[(size_t)q * ccap + slot] = make_uint2(__float_as_uint(val[i]), (uint32_t)(ct * kTileN + (2 * chalf + g) * 32 + i));
+                                ++slot;
+                            }
                         }
-                    } else {
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int g = 0; g < 2; ++g) {
+                    const int cc = 2 * chalf + g;
+                    float val[32];
+                    values(cc, val);
+                    const int c0 = ct * kTileN + cc * 32;
+                    if (q < nqc) {
+                        float* dst = out + (size_t)q * out_stride + c0;
+                        if (c0 + 32 <= nlist && (out_stride & 3) == 0) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (c0 + i < nlist) dst[i] = fmaf(-2.0f, __uint_as_float(v[i]), __ldg(cnorm + c0 + i));
+                            for (int i = 0; i < 32; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(val[i], val[i + 1], val[i + 2], val[i + 3]);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i)
+                                if (c0 + i < nlist) dst[i] = val[i];
+                        }
                     }
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[buf]));
+            }
+            if (et < kTileN) sh->cn[buf ^ 1][et] = cn_next;
+            if (et == 0) sh->epi_stop[buf] = *abort_word;
+            epi_sync();   // the next tile's norms are in place (its buffer was last read two barriers ago)
+            if (sh->epi_stop[buf]) break;
         }
     }
 
@@ -292,7 +376,10 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
                                                           const float* __restrict__ cent, const unsigned* __restrict__ cmax_bits,
                                                           int nlist, int d, int nprobe, int64_t q0,
                                                           int32_t* __restrict__ probe_ids, float* __restrict__ probe_d,
-                                                          int* __restrict__ status) {
+                                                          int* __restrict__ status, const uint2* __restrict__ clist,
+                                                          const int* __restrict__ ccount, int ccap) {
+    // clist != null: the proposals are the (value, cluster) pairs the filtering epilogue kept for this
+    // query instead of a full row; a list that did not fit means: evaluate every cluster exactly.
     extern __shared__ __align__(1024) unsigned char dyn[];
     unsigned long long* buf = reinterpret_cast<unsigned long long*>(dyn);                 // [kTopkCap]
     int* cand = reinterpret_cast<int*>(dyn + (size_t)kTopkCap * 8);                       // [kCandCap]
@@ -307,6 +394,12 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
     const int tid = threadIdx.x;
     const int64_t q = q0 + blockIdx.x;
     const float* row = approx + (size_t)blockIdx.x * nlist;
+    const bool from_list = clist != nullptr;
+    const uint2* cl = clist + (size_t)blockIdx.x * ccap;
+    const int nlisted = from_list ? ccount[blockIdx.x] : 0;
+    const int nsrc = from_list ? min(nlisted, ccap) : nlist;
+    auto src_val = [&](int i) { return from_list ? __uint_as_float(cl[i].x) : row[i]; };
+    auto src_id = [&](int i) { return from_list ? (int)cl[i].y : i; };
 
     float part = 0.0f;
     for (int j = tid; j < d; j += 256) {
@@ -348,19 +441,19 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
         return a;
     };
 
-    bool all_exact = nprobe >= nlist;
+    bool all_exact = nprobe >= nlist || (from_list && (nlisted > ccap || nlisted < nprobe));
     if (!all_exact) {
         // ---- a bound at or above the nprobe-th smallest approximate distance: stream the row
         //      through the buffer, compacting by histogram whenever it could overflow ----
-        if (nlist <= kTopkCap) {
+        if (nsrc <= kTopkCap) {
             // the whole row fits the buffer: every key goes to its own slot, no counting, no barriers
-            for (int c = tid; c < nlist; c += 256) buf[c] = make_key(fmaxf(row[c] + qn, 0.0f), (uint32_t)c);
-            if (tid == 0) cnt = nlist;
+            for (int c = tid; c < nsrc; c += 256) buf[c] = make_key(fmaxf(src_val(c) + qn, 0.0f), (uint32_t)src_id(c));
+            if (tid == 0) cnt = nsrc;
         } else {
-            for (int base = 0; base < nlist; base += 256) {
+            for (int base = 0; base < nsrc; base += 256) {
                 const int c = base + tid;
-                if (c < nlist) {
-                    const unsigned long long key = make_key(fmaxf(row[c] + qn, 0.0f), (uint32_t)c);
+                if (c < nsrc) {
+                    const unsigned long long key = make_key(fmaxf(src_val(c) + qn, 0.0f), (uint32_t)src_id(c));
                     if (key < tau) {
                         if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
                     }
@@ -376,10 +469,10 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
         const float cut = bound + 2.0f * eps;
         __syncthreads();
         // ---- everything under the cut ----
-        for (int c = tid; c < nlist; c += 256) {
-            if (fmaxf(row[c] + qn, 0.0f) <= cut) {
+        for (int c = tid; c < nsrc; c += 256) {
+            if (fmaxf(src_val(c) + qn, 0.0f) <= cut) {
                 const int pos = atomicAdd(&ncand, 1);
-                if (pos < kCandCap) cand[pos] = c;
+                if (pos < kCandCap) cand[pos] = src_id(c);
             }
         }
         __syncthreads();
@@ -415,6 +508,107 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
             probe_ids[q * nprobe + rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
             probe_d[q * nprobe + rank] = __uint_as_float((uint32_t)(key >> 32));
         });
+    }
+}
+
+// One CTA per query: an upper bound of the nprobe-th smallest of the query's `m` sampled values (any m
+// clusters: the value is then an upper bound of the nprobe-th smallest over all clusters), plus twice
+// the error bound of the approximate values, is the cut the filtering epilogue compares with.  Also
+// clears the query's candidate counter.  Values are |c|^2 - 2 q.c (without |q|^2, which is constant
+// per query).  m <= 16 * 256: every thread keeps its values in registers, as order-preserving bits.
+// Two histogram passes of 256 bins (the value range, then the bin that holds the wanted rank) place
+// the bound within 2^-16 of the range above the exact order statistic.
+constexpr int kBoundPerThread = 16;
+__global__ void __launch_bounds__(256) probe_bound_kernel(const float* __restrict__ sample, int m, const float* __restrict__ queries,
+                                                         const unsigned* __restrict__ cmax_bits, int d, int nprobe, int64_t q0,
+                                                         float* __restrict__ cutp, int* __restrict__ ccount) {
+    __shared__ int hist[256];
+    __shared__ int wsum[8];
+    __shared__ unsigned mm[2];
+    __shared__ int found[2];
+    __shared__ float red[8];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int ql = blockIdx.x;
+    const float* row = sample + (size_t)ql * m;
+    uint32_t ob[kBoundPerThread];
+    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+#pragma unroll
+    for (int j = 0; j < kBoundPerThread; ++j) {
+        const int i = tid + 256 * j;
+        ob[j] = i < m ? ordered_bits(row[i]) : 0xFFFFFFFFu;   // beyond the sample: after every real value
+        if (i < m) {
+            lo = min(lo, ob[j]);
+            hi = max(hi, ob[j]);
+        }
+    }
+    float qn = 0.0f;
+    for (int j = tid; j < d; j += 256) {
+        const float x = queries[(q0 + ql) * d + j];
+        qn = fmaf(x, x, qn);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) qn += __shfl_xor_sync(0xFFFFFFFFu, qn, o);
+    lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+    if (tid == 0) {
+        mm[0] = 0xFFFFFFFFu;
+        mm[1] = 0u;
+    }
+    hist[tid] = 0;
+    __syncthreads();
+    if (lane == 0) {
+        red[warp] = qn;
+        atomicMin(&mm[0], lo);
+        atomicMax(&mm[1], hi);
+    }
+    __syncthreads();
+    lo = mm[0];
+    hi = mm[1];
+    uint32_t base = lo;        // first value of the bin range in work
+    uint32_t top = hi;         // every value of interest is <= top
+    int need = nprobe;         // rank wanted among the values >= base
+    for (int pass = 0; pass < 2; ++pass) {
+        const uint32_t range = top - base;
+        int shift = 0;   // smallest shift with (range >> shift) < 256
+        if (range >= 256u) shift = (32 - __clz(range)) - 8;
+#pragma unroll
+        for (int j = 0; j < kBoundPerThread; ++j)
+            if (ob[j] >= base && ob[j] <= top) atomicAdd(&hist[(ob[j] - base) >> shift], 1);
+        __syncthreads();
+        const int v = hist[tid];
+        int incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int x = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += x;
+        }
+        if (lane == 31) wsum[warp] = incl;
+        __syncthreads();
+        int before = 0;
+        for (int w = 0; w < warp; ++w) before += wsum[w];
+        incl += before;
+        if (incl - v < need && need <= incl) {   // exactly one thread: its bin holds the wanted rank
+            found[0] = tid;
+            found[1] = incl - v;
+        }
+        hist[tid] = 0;
+        __syncthreads();
+        const int bin = found[0];
+        need -= found[1];
+        const uint32_t nbase = base + ((uint32_t)bin << shift);
+        const unsigned long long ntop = (unsigned long long)nbase + ((1ull << shift) - 1ull);
+        base = nbase;
+        top = ntop < (unsigned long long)top ? (uint32_t)ntop : top;
+        if (shift == 0) break;   // the bin is a single value (uniform)
+    }
+    if (tid == 0) {
+        qn = 0.0f;
+        for (int i = 0; i < 8; ++i) qn += red[i];
+        const float kth = from_ordered_bits(top);   // at or above the nprobe-th smallest sampled value
+        const float cmax = __uint_as_float(*cmax_bits);
+        const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
+        cutp[ql] = kth + 2.0f * eps + 1e-6f * fabsf(kth);   // the last term: the two sides add |q|^2 in different places
+        ccount[ql] = 0;
     }
 }
 
@@ -464,8 +658,28 @@ cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cuda
     return cudaGetLastError();
 }
 
+constexpr int kSampleMax = 256 * kBoundPerThread;   // clusters of the bound-giving first pass, at most
+constexpr int kListCap = 1024;                      // candidate entries kept per query by the fused epilogue
+
+// Clusters of the first pass: a quarter of them (whole tiles), at most kSampleMax.
+static int sample_clusters(int nlist) {
+    int m = (nlist / 4) / kTileN * kTileN;
+    return m > kSampleMax ? kSampleMax : m;
+}
+
+// Whether the fused path (no [queries][nlist] tile) serves this shape: many clusters, and an expected
+// list (nlist * nprobe / sample, before the widening by the error bound) well under its capacity.
+bool coarse_mma_fused(int nlist, int nprobe) {
+    if (nlist < 8192) return false;
+    return (int64_t)nlist * nprobe / sample_clusters(nlist) <= kListCap / 4;
+}
+
+// Bytes of scratch per query of the fused path: sample row, cut, counter, candidate list.
+size_t coarse_mma_fused_bytes_per_query(int nlist) { return (size_t)sample_clusters(nlist) * 4 + 8 + (size_t)kListCap * 8; }
+
 // Tensor-core filtering of the queries [q0, q0 + nqc): returns cudaErrorNotSupported when the
-// tensor maps cannot be built (the caller then uses the plain kernels).
+// tensor maps cannot be built (the caller then uses the plain kernels).  `tile` is scratch of at
+// least nqc * nlist floats (full-tile path) or nqc * coarse_mma_fused_bytes_per_query() bytes.
 cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe,
                               float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
                               int64_t* launches) {
@@ -475,23 +689,46 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
     const int kblocks = (ix->d + kKBlock - 1) / kKBlock;
     const int qtiles = (nqc + kTileM - 1) / kTileM;
     const int ntile = (ix->nlist + kTileN - 1) / kTileN;
-    int csplit = (2 * ix->sm_count + qtiles - 1) / qtiles;   // about two waves of CTAs
-    if (csplit > ntile) csplit = ntile;
-    if (csplit < 1) csplit = 1;
-    const size_t smem = 1024 + (size_t)(kblocks + kStages) * kTileBytes + sizeof(MmaShared);
+    auto csplit_for = [&](int tiles) {
+        int cs = (2 * ix->sm_count + qtiles - 1) / qtiles;   // about two waves of CTAs
+        if (cs > tiles) cs = tiles;
+        return cs < 1 ? 1 : cs;
+    };
+    int nstages = 12 - kblocks;   // 16 KB tiles: queries + stages within about 200 KB
+    if (nstages > kStages) nstages = kStages;
+    const size_t smem = 1024 + (size_t)(kblocks + nstages) * kTileBytes + sizeof(MmaShared);
     cudaError_t e = cudaFuncSetAttribute(coarse_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const float* cnorm = ix->cnorm;
     const unsigned* cmax = reinterpret_cast<const unsigned*>(reinterpret_cast<const char*>(cnorm) + align_up((size_t)ix->nlist * 4, 256));
-    coarse_mma_kernel<<<dim3(qtiles, csplit), kMmaThreads, smem, st>>>(map_q, map_c, cnorm, nqc, ix->nlist, kblocks, tile, status,
-                                                                       ix->test_fault);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
     const size_t smem2 = (size_t)kTopkCap * 8 + (size_t)kCandCap * 4 + align_up((size_t)ix->d * 4, 16);
     e = cudaFuncSetAttribute(probe_rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
     if (e != cudaSuccess) return e;
+
+    if (coarse_mma_fused(ix->nlist, nprobe) && !ix->test_fault) {
+        // scratch: [nqc][sample] values | [nqc] cuts | [nqc] counters | [nqc][kListCap] (value, cluster)
+        const int nsample = sample_clusters(ix->nlist);
+        float* sample = tile;
+        float* cutp = sample + (size_t)nqc * nsample;
+        int* ccount = reinterpret_cast<int*>(cutp + nqc);
+        uint2* clist = reinterpret_cast<uint2*>(ccount + nqc);   // 8-byte aligned: 2 nqc words of cuts and counters before it
+        const int stile = nsample / kTileN;
+        coarse_mma_kernel<<<dim3(qtiles, csplit_for(stile)), kMmaThreads, smem, st>>>(
+            map_q, map_c, cnorm, nqc, ix->nlist, kblocks, sample, status, 0, stile, nsample, nullptr, nullptr, nullptr, 0, nstages);
+        probe_bound_kernel<<<nqc, 256, 0, st>>>(sample, nsample, queries, cmax, ix->d, nprobe, q0, cutp, ccount);
+        coarse_mma_kernel<<<dim3(qtiles, csplit_for(ntile)), kMmaThreads, smem, st>>>(
+            map_q, map_c, cnorm, nqc, ix->nlist, kblocks, nullptr, status, 0, ntile, 0, cutp, ccount, clist, kListCap, nstages);
+        probe_rerank_kernel<<<nqc, 256, smem2, st>>>(nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
+                                                      probe_d, status, clist, ccount, kListCap);
+        *launches += 4;
+        return cudaGetLastError();
+    }
+    coarse_mma_kernel<<<dim3(qtiles, csplit_for(ntile)), kMmaThreads, smem, st>>>(map_q, map_c, cnorm, nqc, ix->nlist, kblocks, tile, status,
+                                                                                 ix->test_fault, ntile, ix->nlist, nullptr, nullptr, nullptr, 0, nstages);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     probe_rerank_kernel<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
-                                                  probe_d, status);
+                                                  probe_d, status, nullptr, nullptr, 0);
     *launches += 2;
     return cudaGetLastError();
 }

@@ -125,6 +125,8 @@ bool rot_supported(int nsub, int dsub);
 // Tensor-core filtering (coarse_mma.cu).
 bool coarse_mma_supported(int d, int nlist);
 size_t coarse_mma_derived_bytes(int nlist);
+bool coarse_mma_fused(int nlist, int nprobe);
+size_t coarse_mma_fused_bytes_per_query(int nlist);
 cudaError_t launch_entry_map(const ivfpq_index* ix, const uint8_t* codes, cudaStream_t st);
 cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st);
 cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe,
@@ -139,6 +141,8 @@ cudaError_t launch_entry_stats(const ivfpq_index* ix, const uint8_t* codes, cons
 cudaError_t launch_negate(const float* in, float* out, int64_t n, cudaStream_t st);
 cudaError_t launch_thresholds(const float* queries, int64_t nq, int nsub, const ivfpq_threshold_model_t* m,
                               float* radius, cudaStream_t st);
+cudaError_t launch_thresholds_knn(const ivfpq_index* ix, const float* queries, int64_t nq, const int32_t* probe0, int kth,
+                                  int degree, const float* coef, float* radius, int* status, cudaStream_t st);
 cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws, cudaStream_t st,
                         int64_t* launches);
 

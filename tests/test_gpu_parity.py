@@ -111,6 +111,52 @@ def test_probe_lists_many_clusters():
         lib.ivfpq_index_free(h)
 
 
+def test_probe_lists_fused_selection_large_nlist():
+    """8192 clusters or more with few probes: the filtering epilogue keeps only the values under a cut
+    taken from the first 1024 clusters instead of writing full rows (probe counts 1..64); 65 probes
+    and more go through the full rows.  Same probe lists, bit for bit, either way."""
+    wl = Workload(small_cfg("c1", n=40_000, d=64, nsub=8, dsub=8, ncomp=500, nlist=9000, nq=301, chunk=16384,
+                            kmeans_iters=2))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        q = dev(wl.queries)
+        for nprobe in (1, 7, 32, 64, 65, 200):
+            pid, pd = lib.ivfpq_debug_probes(h, q, nprobe)
+            opid, opd = oracle.coarse(wl.index, wl.queries, nprobe)
+            check_status(h)
+            assert np.array_equal(host(pid), opid)
+            assert np.array_equal(host(pd).view(np.uint32), opd.view(np.uint32))
+    finally:
+        lib.ivfpq_index_free(h)
+
+
+@pytest.mark.parametrize("nlist", [300, 8500])
+def test_probe_lists_large_norms_and_near_ties(nlist):
+    """Aimed at the error bound of the tensor-core proposal: coordinates around 1e4 with unit spread
+    (the TF32 products are off by far more than the distances differ, so nearly every cluster falls
+    under the cut), duplicated centroids (exact ties, decided by cluster id) and queries much shorter
+    than the centroids.  A loose bound would drop a true probe; the lists must stay bit-equal."""
+    rng = np.random.default_rng(nlist)
+    d = 64
+    idx, base = lossless_toy_index(seed=9, n=2 * nlist, nlist=nlist, nsub=8, dsub=8, ksub=16, spread=1.0)
+    cent = (idx.coarse_centroids + 1.0e4).astype(F32)
+    cent[1::7] = cent[0:-1:7][: len(cent[1::7])]           # duplicates: exact ties
+    idx.coarse_centroids = cent
+    h = lib.ivfpq_index_load(idx)
+    try:
+        q_far = (cent[rng.integers(0, nlist, 96)] + rng.standard_normal((96, d))).astype(F32)
+        q_short = (rng.standard_normal((32, d)) * 1.0e2).astype(F32)      # |q| about 1e-2 of |c|
+        q = np.concatenate([q_far, q_short])
+        for nprobe in (1, 8, 33):
+            pid, pd = lib.ivfpq_debug_probes(h, dev(q), nprobe)
+            opid, opd = oracle.coarse(idx, q, nprobe)
+            check_status(h)
+            assert np.array_equal(host(pid), opid)
+            assert np.array_equal(host(pd).view(np.uint32), opd.view(np.uint32))
+    finally:
+        lib.ivfpq_index_free(h)
+
+
 def test_probe_all_lists(loaded):
     wl, h = loaded["small"]
     pid, pd = lib.ivfpq_debug_probes(h, dev(wl.queries), wl.index.nlist)

@@ -112,3 +112,40 @@ def test_threshold_errors(wl_small, wl_pq2):
     finally:
         lib.ivfpq_index_free(h4)
         lib.ivfpq_index_free(h2)
+
+
+@pytest.mark.parametrize("shape", ["16x8", "50x4", "12x2", "10x3"])
+def test_kth_nearest_entry_thresholds_bit_equal(shape):
+    """Thresholds from the kth-nearest codebook entry (any subspace width): the CUDA kernel and the
+    oracle take the same fp32 steps, so the radii are bit-equal; they then drive the sparse search."""
+    from conftest import Workload, small_cfg
+    from parity import assert_topk_parity
+    cfgs = {"16x8": ("c1", dict(n=12_000, ncomp=120, nlist=40, nq=70)),
+            "50x4": ("c4", dict(n=12_000, ncomp=120, nlist=40, nq=70)),
+            "12x2": ("c3", dict(n=8_000, d=24, nsub=12, dsub=2, ncomp=100, nlist=30, nq=70)),
+            "10x3": ("c4", dict(n=6_000, d=30, nsub=10, dsub=3, ncomp=80, nlist=23, nq=50))}
+    base, kw = cfgs[shape]
+    wl = Workload(small_cfg(base, chunk=8192, kmeans_iters=3, **kw))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        rng = np.random.default_rng(3)
+        q = torch.from_numpy(wl.queries).cuda()
+        for kth, degree in ((1, 1), (64, 1), (wl.index.ksub, 0), (17, 3)):
+            coef = (rng.standard_normal((wl.index.nsub, degree + 1)) * 0.3).astype(np.float32)
+            coef[:, 0] += 0.5
+            if degree == 1 and kth == 64:
+                coef[:] = np.array([0.0, 1.0], np.float32)     # the kth-nearest-entry distance itself
+            g = lib.ivfpq_query_thresholds_knn(h, q, kth, torch.from_numpy(coef).cuda())
+            assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
+            o = oracle.thresholds_knn(wl.index, wl.queries, kth, coef)
+            assert np.array_equal(g.cpu().numpy().view(np.uint32), o.view(np.uint32)), (kth, degree)
+        # the identity radii at rank 64 feed the sparse search in per-query mode
+        ident = torch.tensor([[0.0, 1.0]] * wl.index.nsub, device="cuda")
+        d, i = lib.ivfpq_search_sparse(h, q, 5, lib.ivfpq_query_thresholds_knn(h, q, 64, ident), 30, scale=0.9)
+        rad = oracle.thresholds_knn(wl.index, wl.queries, 64, np.tile(np.array([[0.0, 1.0]], np.float32), (wl.index.nsub, 1)))
+        oo = oracle.search(wl.index, wl.queries, 5, 30, radius=rad, scale=0.9)
+        assert_topk_parity(d.cpu().numpy(), i.cpu().numpy(), oo["dist"], oo["ids"])
+        with pytest.raises(lib.IvfpqError):
+            lib.ivfpq_query_thresholds_knn(h, q, 0, torch.zeros((wl.index.nsub, 2), device="cuda"))
+    finally:
+        lib.ivfpq_index_free(h)

@@ -87,6 +87,8 @@ def test_load_rejects_bad_arguments_before_any_cuda_call(L):
     assert L.ivfpq_last_launch_count(None) == 0
     assert L.ivfpq_probe_static(None, None, 1, 1, None, None, None) == lib.IVFPQ_ERR_INVALID_ARGUMENT
     assert L.ivfpq_query_thresholds(None, None, 1, None, None, None) == lib.IVFPQ_ERR_INVALID_ARGUMENT
+    assert L.ivfpq_query_thresholds_knn(None, None, 1, 1, 1, None, None, None, 0, None) == lib.IVFPQ_ERR_INVALID_ARGUMENT
+    assert L.ivfpq_static_status is not None
     assert L.ivfpq_entry_stats(None, None, None, 1, None, 1, None, None, None, None) == lib.IVFPQ_ERR_INVALID_ARGUMENT
 
 
