@@ -140,16 +140,19 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
     const bool mma_shape = !ip && ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
                            (reinterpret_cast<uintptr_t>(ix->cent) & 15) == 0;
     const int64_t qchunk_row = qchunk;   // queries whose full rows fit the scratch region (the plain kernels need those)
-    bool mma = mma_shape;
+    bool mma = mma_shape, fused = false;
     if (mma && coarse_mma_fused(ix->nlist, nprobe) && !ix->test_fault) {
-        // the fused path needs far less scratch per query than a full row: larger query chunks in the same region
-        const int64_t fit = (int64_t)(((size_t)qchunk * ix->nlist * 4 - 16) / coarse_mma_fused_bytes_per_query(ix->nlist));
-        if (fit > qchunk) qchunk = fit < nq ? fit : nq;
+        // the fused path needs another amount of scratch per query than a full row: its own chunking of the same region
+        const int64_t fit = (int64_t)(((size_t)qchunk * ix->nlist * 4) / coarse_mma_fused_bytes_per_query(ix->nlist));
+        if (fit >= 1) {
+            qchunk = fit < nq ? fit : nq;   // more queries per chunk than full rows would allow, or fewer
+            fused = true;
+        }
     }
     for (int64_t q0 = 0; q0 < nq; q0 += qchunk) {
         int nqc = (int)((nq - q0 < qchunk) ? (nq - q0) : qchunk);
         if (mma) {
-            const cudaError_t e = launch_coarse_mma(ix, queries, q0, nqc, nprobe, coarse_tile, probe_ids, probe_d, status, st, launches);
+            const cudaError_t e = launch_coarse_mma(ix, queries, q0, nqc, nprobe, fused, coarse_tile, probe_ids, probe_d, status, st, launches);
             if (e == cudaSuccess) continue;
             if (e != cudaErrorNotSupported) return e;
             mma = false;   // the tensor maps could not be built: the plain kernels, in chunks of full rows

@@ -129,7 +129,7 @@ bool coarse_mma_fused(int nlist, int nprobe);
 size_t coarse_mma_fused_bytes_per_query(int nlist);
 cudaError_t launch_entry_map(const ivfpq_index* ix, const uint8_t* codes, cudaStream_t st);
 cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st);
-cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe,
+cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe, bool fused,
                               float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
                               int64_t* launches);
 cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,

@@ -113,8 +113,9 @@ def test_probe_lists_many_clusters():
 
 def test_probe_lists_fused_selection_large_nlist():
     """8192 clusters or more with few probes: the filtering epilogue keeps only the values under a cut
-    taken from the first 1024 clusters instead of writing full rows (probe counts 1..64); 65 probes
-    and more go through the full rows.  Same probe lists, bit for bit, either way."""
+    taken from the first quarter of the clusters instead of writing full rows; many probes go through
+    the full rows.  Same probe lists, bit for bit, either way, also for batches of one and three
+    queries (their scratch is chunked differently)."""
     wl = Workload(small_cfg("c1", n=40_000, d=64, nsub=8, dsub=8, ncomp=500, nlist=9000, nq=301, chunk=16384,
                             kmeans_iters=2))
     h = lib.ivfpq_index_load(wl.index)
@@ -126,11 +127,15 @@ def test_probe_lists_fused_selection_large_nlist():
             check_status(h)
             assert np.array_equal(host(pid), opid)
             assert np.array_equal(host(pd).view(np.uint32), opd.view(np.uint32))
+            for n in (1, 3):
+                pid, pd = lib.ivfpq_debug_probes(h, q[:n].contiguous(), nprobe)
+                check_status(h)
+                assert np.array_equal(host(pid), opid[:n])
     finally:
         lib.ivfpq_index_free(h)
 
 
-@pytest.mark.parametrize("nlist", [300, 8500])
+@pytest.mark.parametrize("nlist", [300, 1100, 8500])
 def test_probe_lists_large_norms_and_near_ties(nlist):
     """Aimed at the error bound of the tensor-core proposal: coordinates around 1e4 with unit spread
     (the TF32 products are off by far more than the distances differ, so nearly every cluster falls
