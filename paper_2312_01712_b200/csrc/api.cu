@@ -113,7 +113,9 @@ int run_search(SearchArgs a, void* workspace, size_t workspace_bytes, void* stre
         ix->ev_ready = true;
     }
     // keep_status: a later slice of one batch adds its flags to those of the earlier slices
+    // status block: word 0 = device flags, word 1 = work counter of the persistent scan kernels
     if (!keep_status && cudaMemsetAsync(ws + wl.status_off, 0, 16, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
+    if (keep_status && cudaMemsetAsync(ws + wl.status_off + 4, 0, 12, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
     if (timed && cudaEventRecord(ix->ev[0], st) != cudaSuccess) return IVFPQ_ERR_CUDA;
     int32_t* probe_ids = reinterpret_cast<int32_t*>(ws + wl.probe_ids_off);
     float* probe_d = reinterpret_cast<float*>(ws + wl.probe_d_off);
@@ -239,6 +241,8 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
         const char* kind = getenv("IVFPQ_SCAN_KERNEL");
         if (kind && strcmp(kind, "warps16") == 0) ix->pers_warps = 16;
         if (kind && strcmp(kind, "warps32") == 0) ix->pers_warps = 32;
+        const char* rk = getenv("IVFPQ_ROT_KERNEL");
+        ix->rot_pair = (rk && strcmp(rk, "pair") == 0) ? 1 : 0;
     }
     for (int i = 0; i < 3; ++i) ix->gw[i] = dl.rot ? dl.gw[i] : 0;
     ix->block_bytes = dl.block_bytes;

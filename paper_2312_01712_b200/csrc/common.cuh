@@ -43,6 +43,7 @@ struct ivfpq_index {
     // the lane's own visiting order, codebook copied entry-major per group
     int32_t pers_warps;       // 16 x 8 shape: warps per CTA of the persistent kernel (16: short lists, 32: long lists)
     int32_t rot;              // 1: rotated layout in use
+    int32_t rot_pair;         // wide rotated shapes: 1 = two clusters per table-build pass (scan_rot.cu)
     int32_t gw[3];            // group widths, largest first, 0 = unused
     int32_t block_bytes;      // bytes of one 32-point code block in the rotated layout
     const float* cbt;         // [group][entry 0..255][column][dsub]

@@ -513,6 +513,7 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     sp.out_ids = a.out_ids;
     sp.partial = reinterpret_cast<unsigned long long*>(ws + wl.partial_off);
     sp.status = reinterpret_cast<int*>(ws + wl.status_off);
+    sp.work = sp.status + 1;
     sp.masks = a.masks;
     sp.visit_count = a.visit_count;
     sp.visit_stride = a.visit_stride;

@@ -159,6 +159,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(a);
     int* cnt_p = reinterpret_cast<int*>(a + 8);
     int* ntrans_p = cnt_p + 1;
+    int* next_p = cnt_p + 2;   // the item this CTA takes next
     a += 32;
     int* hist_p = reinterpret_cast<int*>(a);
     a += kQuickWords * 4;
@@ -245,7 +246,10 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
 
     topk_quick_init<kNT>(hist_p);  // contains a barrier: the shared half of the codebook is complete too
 
-    for (int64_t item = blockIdx.x; item < nitems; item += gridDim.x) {
+    // Items beyond the first come from a global counter (lists differ in length: a fixed stride
+    // leaves the CTAs finishing at different times); the draw is made at the start of an item and read
+    // at its end.
+    for (int64_t item = blockIdx.x; item < nitems; item = *next_p) {
         const int64_t q = item / p.nsplit;
         const int split = (int)(item % p.nsplit);
         const int np_item = (p.nprobe - split + p.nsplit - 1) / p.nsplit;  // probes split, split + nsplit, ...
@@ -258,6 +262,8 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
             *cnt_p = 0;
             *ntrans_p = 0;
             *tau_p = kKeyPad;
+        } else if (tid == 65) {
+            *next_p = (int)gridDim.x + atomicAdd(p.work, 1);
         }
         if (DBG && tid == 96) fill_visit_prefix(p, q, vprefix);
         float P = 0.0f, thr = 0.0f;

@@ -35,6 +35,7 @@ struct ScanParams {
     int32_t* out_ids;
     unsigned long long* partial;
     int* status;
+    int* work;   // zeroed per launch: the persistent kernels draw their items beyond the first from it
     // stage dumps (DBG instantiations only)
     uint32_t* masks;
     int64_t* visit_count;

@@ -15,6 +15,8 @@
 // The table is built with lanes running over the columns of a row (not over entries), reading
 // the codebook from an entry-major copy made at load time, so both the codebook loads and the
 // table stores are contiguous / conflict-free.
+#include <type_traits>
+
 #include "common.cuh"
 #include "scan_common.cuh"
 #include "topk.cuh"
@@ -35,8 +37,11 @@ __host__ __device__ constexpr int lane_bytes(int w) { return w >= 16 ? w : (w ==
 // 256 bytes, [32 columns of group 0 | 32 columns of group 1], at a fixed address of the CTA's
 // shared window, so that a look-up address is {code, column offset} put together by one byte
 // permute and the base is an immediate of the load.
-constexpr uint32_t kPairWin = 0x5000;          // shared-window address of the paired tables (64 KB)
 constexpr int kPairRowFloats = 64;
+// shared-window address of the paired tables (64 KB per cluster): behind the auxiliary data, which is
+// larger for the instance that works on two clusters at a time (4096 candidate slots, two residuals)
+__host__ __device__ constexpr uint32_t pair_win(int nc) { return nc == 2 ? 0xA000u : 0x5000u; }
+__host__ __device__ constexpr int cand_cap(int nc) { return nc == 2 ? 2 * kTopkCap : kTopkCap; }
 
 template <int W0, int W1, int W2>
 struct Groups {
@@ -61,77 +66,90 @@ struct Groups {
     }
 };
 
-// Bytes in front of the tables: candidate keys, residual, thresholds, counters, histogram.
-__host__ __device__ inline size_t rot_aux_bytes(int d) {
-    return (size_t)kTopkCap * 8 + align_up((size_t)d * 4, 16) + IVFPQ_MAX_NSUB * 4 + 32 + kTopkHistInts * 4;
+// Bytes in front of the tables: candidate keys, residual(s), thresholds, counters, histogram.
+__host__ __device__ inline size_t rot_aux_bytes(int d, int nc) {
+    return (size_t)cand_cap(nc) * 8 + nc * align_up((size_t)d * 4, 16) + IVFPQ_MAX_NSUB * 4 + 32 + kTopkHistInts * 4;
 }
 
 // Dynamic shared memory of a launch.  Paired layout: everything up to the fixed table address
 // (whatever the window offset of the allocation turns out to be), the tables, the debug area.
-__host__ __device__ inline size_t rot_smem_bytes(bool paired, int lut_floats, int d, int nprobe, bool dbg) {
-    size_t b = paired ? (size_t)kPairWin : rot_aux_bytes(d);
-    b += (size_t)lut_floats * 4;
-    if (dbg) b += IVFPQ_MAX_NSUB * 8 * 4 + (size_t)(nprobe + 1) * 8;
+__host__ __device__ inline size_t rot_smem_bytes(bool paired, int lut_floats, int d, int nprobe, bool dbg, int nc) {
+    size_t b = paired ? (size_t)pair_win(nc) : rot_aux_bytes(d, nc);
+    b += (size_t)nc * lut_floats * 4;
+    if (dbg) b += (size_t)nc * IVFPQ_MAX_NSUB * 8 * 4 + (size_t)(nprobe + 1) * 8;
     return b;
 }
 
-// Table of one group for one (query, cluster): thread t owns column c = t & (W-1) and the
-// entries u, u + NT/W, ... with u = t / W.
-template <int W, int DSUB, int NT, bool DBG, int SCORE_T, int RS = row_stride(W)>
-__device__ __forceinline__ void build_group(float* __restrict__ lutg, const float* __restrict__ cbt_g,
-                                            const float* __restrict__ res_g, const float* __restrict__ r2_g,
-                                            int ksub, bool dense, int score, float P, uint32_t* hitmask_g) {
+// Table of one group for NC (query, cluster) pairs of the same query: thread t owns column
+// c = t & (W-1) and the entries u, u + NT/W, ... with u = t / W.  Every codebook entry is loaded once
+// and measured against the residuals of all NC clusters (the codebook comes through L2: with two
+// clusters per pass its traffic per table halves).  lut_step / res_step / hm_step: distance between
+// the clusters' tables, residuals and stage-dump masks.
+template <int W, int DSUB, int NT, bool DBG, int SCORE_T, int NC, int RS = row_stride(W)>
+__device__ __forceinline__ void build_group(float* __restrict__ lutg, int lut_step, const float* __restrict__ cbt_g,
+                                            const float* __restrict__ res_g, int res_step, const float* __restrict__ r2_g,
+                                            int ksub, bool dense, int score, float P, uint32_t* hitmask_g, int hm_step) {
     constexpr int EP = NT / W;      // entries per pass
     constexpr int NCOPY = (RS == kPairRowFloats ? 32 : RS) / W;   // copies within the group's 32 (or w) columns
     const int t = threadIdx.x;
     const int c = t & (W - 1);
     const int u = t / W;
     const int usub = (t & 31) / W;  // which of the warp's entries this lane works on
-    float r[DSUB];
+    float r[NC][DSUB];
 #pragma unroll
-    for (int j = 0; j < DSUB; ++j) r[j] = res_g[c * DSUB + j];
+    for (int k = 0; k < NC; ++k)
+#pragma unroll
+        for (int j = 0; j < DSUB; ++j) r[k][j] = res_g[k * res_step + c * DSUB + j];
     const float thr = r2_g[c];
 #pragma unroll 2
     for (int e = u; e < 256; e += EP) {
-        float d2 = 0.0f;
-        bool hit = false;
+        float d2[NC];
+        bool hit[NC];
+#pragma unroll
+        for (int k = 0; k < NC; ++k) {
+            d2[k] = 0.0f;
+            hit[k] = false;
+        }
         if (e < ksub) {
             const float* ent = cbt_g + ((size_t)e * W + c) * DSUB;
+            float ev[DSUB];
             if constexpr (DSUB % 4 == 0) {
 #pragma unroll
                 for (int j4 = 0; j4 < DSUB / 4; ++j4) {
-                    const float4 ev = __ldg(reinterpret_cast<const float4*>(ent) + j4);
-                    float tt;
-                    tt = __fsub_rn(r[4 * j4 + 0], ev.x); d2 = __fmaf_rn(tt, tt, d2);
-                    tt = __fsub_rn(r[4 * j4 + 1], ev.y); d2 = __fmaf_rn(tt, tt, d2);
-                    tt = __fsub_rn(r[4 * j4 + 2], ev.z); d2 = __fmaf_rn(tt, tt, d2);
-                    tt = __fsub_rn(r[4 * j4 + 3], ev.w); d2 = __fmaf_rn(tt, tt, d2);
+                    const float4 x = __ldg(reinterpret_cast<const float4*>(ent) + j4);
+                    ev[4 * j4] = x.x; ev[4 * j4 + 1] = x.y; ev[4 * j4 + 2] = x.z; ev[4 * j4 + 3] = x.w;
                 }
             } else if constexpr (DSUB % 2 == 0) {
 #pragma unroll
                 for (int j2 = 0; j2 < DSUB / 2; ++j2) {
-                    const float2 ev = __ldg(reinterpret_cast<const float2*>(ent) + j2);
-                    float tt;
-                    tt = __fsub_rn(r[2 * j2 + 0], ev.x); d2 = __fmaf_rn(tt, tt, d2);
-                    tt = __fsub_rn(r[2 * j2 + 1], ev.y); d2 = __fmaf_rn(tt, tt, d2);
+                    const float2 x = __ldg(reinterpret_cast<const float2*>(ent) + j2);
+                    ev[2 * j2] = x.x; ev[2 * j2 + 1] = x.y;
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < DSUB; ++j) {
-                    float tt = __fsub_rn(r[j], __ldg(ent + j));
-                    d2 = __fmaf_rn(tt, tt, d2);
-                }
+                for (int j = 0; j < DSUB; ++j) ev[j] = __ldg(ent + j);
             }
-            hit = dense || d2 <= thr;
-        }
-        const float val = table_value<SCORE_T>(score, hit, d2, thr, P);
-        float* row = lutg + e * RS + c;
 #pragma unroll
-        for (int it = 0; it < NCOPY; ++it) {
-            const int copy = (it + usub) & (NCOPY - 1);  // lanes of a warp write different columns
-            row[copy * W] = val;
+            for (int k = 0; k < NC; ++k) {
+#pragma unroll
+                for (int j = 0; j < DSUB; ++j) {
+                    const float tt = __fsub_rn(r[k][j], ev[j]);
+                    d2[k] = __fmaf_rn(tt, tt, d2[k]);
+                }
+                hit[k] = dense || d2[k] <= thr;
+            }
         }
-        if (DBG && hit) atomicOr(&hitmask_g[c * 8 + (e >> 5)], 1u << (e & 31));
+#pragma unroll
+        for (int k = 0; k < NC; ++k) {
+            const float val = table_value<SCORE_T>(score, hit[k], d2[k], thr, P);
+            float* row = lutg + k * lut_step + e * RS + c;
+#pragma unroll
+            for (int it = 0; it < NCOPY; ++it) {
+                const int copy = (it + usub) & (NCOPY - 1);  // lanes of a warp write different columns
+                row[copy * W] = val;
+            }
+            if (DBG && hit[k]) atomicOr(&hitmask_g[k * hm_step + c * 8 + (e >> 5)], 1u << (e & 31));
+        }
     }
 }
 
@@ -156,24 +174,25 @@ __device__ __forceinline__ void gather_group(const float* __restrict__ lutg, con
 // (lane ^ i) * 4 of the same four steps; T = the byte of both that belongs to this step, G = group.
 // The permute builds {0, 0, code, column offset} (the zero bytes are the replicated sign of the
 // column offset, which is below 128); the table address is the immediate.
-template <int T, int G>
+template <int T, int BASE>
 __device__ __forceinline__ float pair_gather(uint32_t word, uint32_t pack) {
     uint32_t addr;
     float v;
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(addr) : "r"(word), "r"(pack), "n"(((12 + T) << 12) | ((12 + T) << 8) | (T << 4) | (4 + T)));
-    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"((int)kPairWin + G * 128) : "memory");
+    asm volatile("ld.shared.f32 %0, [%1+%2];" : "=f"(v) : "r"(addr), "n"(BASE) : "memory");
     return v;
 }
 
-// Table values of NW code words (4 NW subspaces of group G) added to two running sums.
-template <int NW, int G>
+// Table values of NW code words (4 NW subspaces of one group, whose 32 columns start at the
+// shared-window address BASE) added to two running sums.
+template <int NW, int BASE>
 __device__ __forceinline__ void pair_gather_words(const uint32_t* words, const uint32_t* pk, float& a0, float& a1) {
 #pragma unroll
     for (int j = 0; j < NW; ++j) {
-        a0 += pair_gather<0, G>(words[j], pk[j]);
-        a1 += pair_gather<1, G>(words[j], pk[j]);
-        a0 += pair_gather<2, G>(words[j], pk[j]);
-        a1 += pair_gather<3, G>(words[j], pk[j]);
+        a0 += pair_gather<0, BASE>(words[j], pk[j]);
+        a1 += pair_gather<1, BASE>(words[j], pk[j]);
+        a0 += pair_gather<2, BASE>(words[j], pk[j]);
+        a1 += pair_gather<3, BASE>(words[j], pk[j]);
     }
 }
 
@@ -210,13 +229,20 @@ __device__ __forceinline__ void load_group_codes(const unsigned char* __restrict
     }
 }
 
-template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T>
+// NC = clusters per phase: 1 (one table at a time) or 2 (1024 threads, one CTA per SM; the tables of
+// two probed clusters are built in one pass over the codebook, then both lists are scanned as one
+// sequence of blocks).
+template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T, int NC>
 __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const ScanParams p) {
     using GR = Groups<W0, W1, W2>;
     constexpr int kWarps = NT / 32;
+    constexpr int kCapN = cand_cap(NC);
+    constexpr uint32_t kWin = pair_win(NC);
+    // bytes between the tables of two clusters (the immediate bases of the paired look-ups follow from it)
+    constexpr int kSetBytes = ((GR::kLutFloats * 4 + 255) / 256) * 256;
     // A warp stops after the block in which one of its candidates landed at or beyond the soft limit
     // (at most 32 more per warp): the buffer is then reduced to the k smallest at the next barrier.
-    constexpr int kSoft = kTopkCap - 32 * kWarps;
+    constexpr int kSoft = kCapN - 32 * kWarps;
     static_assert(IVFPQ_MAX_K < kSoft, "candidate buffer too small for the soft limit");
     extern __shared__ __align__(16) unsigned char smem[];
     const int nsub = GR::kNsub;
@@ -225,27 +251,29 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
     const int tid = threadIdx.x;
     const int lane = tid & 31;
     const int warp = tid >> 5;
+    const int dpad = (int)(align_up((size_t)d * 4, 16) / 4);
 
-    // candidate keys | residual | thresholds | counters | histogram | tables | debug area; in the
-    // paired layout the tables start at the fixed window address kPairWin
+    // candidate keys | residual(s) | thresholds | counters | histogram | tables | debug area; in the
+    // paired layout the tables start at the fixed window address kWin
     unsigned long long* kbuf = reinterpret_cast<unsigned long long*>(smem);
-    float* res = reinterpret_cast<float*>(smem + (size_t)kTopkCap * 8);
-    float* r2 = res + align_up((size_t)d * 4, 16) / 4;
+    float* res = reinterpret_cast<float*>(smem + (size_t)kCapN * 8);   // [NC][dpad]
+    float* r2 = res + NC * dpad;
     unsigned long long* tau_p = reinterpret_cast<unsigned long long*>(r2 + IVFPQ_MAX_NSUB);
     int* cnt_p = reinterpret_cast<int*>(tau_p + 1);
     int* hist_p = reinterpret_cast<int*>(tau_p + 4);
-    size_t lut_at = rot_aux_bytes(d);
+    size_t lut_at = rot_aux_bytes(d, NC);
     if constexpr (GR::kPaired) {
         const uint32_t win = (uint32_t)__cvta_generic_to_shared(smem);
-        if (win + lut_at > kPairWin) {   // uniform: the layout does not fit this window offset
+        if (win + lut_at > kWin) {   // uniform: the layout does not fit this window offset
             if (tid == 0) atomicOr(p.status, kFlagLayout);
             return;
         }
-        lut_at = kPairWin - win;
+        lut_at = kWin - win;
     }
-    float* lut = reinterpret_cast<float*>(smem + lut_at);
-    uint32_t* hitmask = reinterpret_cast<uint32_t*>(lut + GR::kLutFloats);             // DBG only
-    long long* vprefix = reinterpret_cast<long long*>(hitmask + IVFPQ_MAX_NSUB * 8);   // DBG only
+    float* lut = reinterpret_cast<float*>(smem + lut_at);                                           // [NC] sets of kSetBytes
+    uint32_t* hitmask = reinterpret_cast<uint32_t*>(smem + lut_at + (size_t)NC * kSetBytes);       // DBG only: [NC][64][8]
+    long long* vprefix = reinterpret_cast<long long*>(hitmask + NC * IVFPQ_MAX_NSUB * 8);           // DBG only
+    constexpr int kSetFloats = kSetBytes / 4;
     // paired layout: column offsets (lane ^ i) * 4 of the 32 steps, four per register
     uint32_t pk[GR::kPaired ? 8 : 1];
     if constexpr (GR::kPaired) {
@@ -291,51 +319,80 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
         }
     }
 
-    for (int pi = split; pi < p.nprobe; pi += p.nsplit) {
-        const int c = p.probe_ids[q * p.nprobe + pi];
-        if (c < 0 || c >= p.nlist) {
-            if (tid == 0) atomicOr(p.status, kFlagBadList);
-            continue;
+    for (int pi0 = split; pi0 < p.nprobe; pi0 += p.nsplit * NC) {
+        // ---- the clusters of this phase; an invalid id leaves an empty list behind ----
+        int cl[NC];
+        int64_t p0[NC], len[NC], b0[NC], nblk[NC];
+#pragma unroll
+        for (int k = 0; k < NC; ++k) {
+            const int pi = pi0 + k * p.nsplit;
+            cl[k] = -1;
+            p0[k] = len[k] = b0[k] = nblk[k] = 0;
+            if (pi < p.nprobe) {
+                const int c = p.probe_ids[q * p.nprobe + pi];
+                if (c < 0 || c >= p.nlist) {
+                    if (tid == 0) atomicOr(p.status, kFlagBadList);
+                } else {
+                    cl[k] = c;
+                    p0[k] = p.list_off[c];
+                    len[k] = p.list_off[c + 1] - p0[k];
+                    b0[k] = p.list_blk[c];
+                    nblk[k] = p.list_blk[c + 1] - b0[k];
+                    if (nblk[k] != (len[k] + kPointsPerBlock - 1) / kPointsPerBlock || len[k] < 0) {
+                        if (tid == 0) atomicOr(p.status, kFlagBadList);
+                        len[k] = nblk[k] = 0;
+                    }
+                }
+            }
         }
-        // (the barrier that ended the previous cluster's scan makes the tables and `res` free)
-        for (int j = tid; j < d; j += NT) res[j] = __fsub_rn(p.queries[q * d + j], p.cent[(int64_t)c * d + j]);
+        // (the barrier that ended the previous phase's scan makes the tables and `res` free)
+#pragma unroll
+        for (int k = 0; k < NC; ++k) {
+            const int c = cl[k] >= 0 ? cl[k] : 0;   // a table is built for every slot; an empty slot is never scanned
+            for (int j = tid; j < d; j += NT) res[k * dpad + j] = __fsub_rn(p.queries[q * d + j], p.cent[(int64_t)c * d + j]);
+        }
         if (DBG)
-            for (int i = tid; i < IVFPQ_MAX_NSUB * 8; i += NT) hitmask[i] = 0;
+            for (int i = tid; i < NC * IVFPQ_MAX_NSUB * 8; i += NT) hitmask[i] = 0;
         __syncthreads();
 
-        // ---- selective tables, one per group ----
-        build_group<W0, DSUB, NT, DBG, SCORE_T, GR::stride(0)>(lut, p.cbt, res, r2, ksub, p.dense, p.score, P, hitmask);
+        // ---- selective tables, one per group and cluster ----
+        build_group<W0, DSUB, NT, DBG, SCORE_T, NC, GR::stride(0)>(lut, kSetFloats, p.cbt, res, dpad, r2, ksub, p.dense, p.score, P,
+                                                                  hitmask, IVFPQ_MAX_NSUB * 8);
         if constexpr (W1 > 0)
-            build_group<W1, DSUB, NT, DBG, SCORE_T, GR::stride(1)>(lut + GR::lut_off(1), p.cbt + (size_t)GR::s0(1) * 256 * DSUB,
-                                           res + GR::s0(1) * DSUB, r2 + GR::s0(1), ksub, p.dense, p.score, P,
-                                           hitmask + GR::s0(1) * 8);
+            build_group<W1, DSUB, NT, DBG, SCORE_T, NC, GR::stride(1)>(lut + GR::lut_off(1), kSetFloats,
+                                                                      p.cbt + (size_t)GR::s0(1) * 256 * DSUB, res + GR::s0(1) * DSUB, dpad,
+                                                                      r2 + GR::s0(1), ksub, p.dense, p.score, P,
+                                                                      hitmask + GR::s0(1) * 8, IVFPQ_MAX_NSUB * 8);
         if constexpr (W2 > 0)
-            build_group<W2, DSUB, NT, DBG, SCORE_T>(lut + GR::lut_off(2), p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
-                                           res + GR::s0(2) * DSUB, r2 + GR::s0(2), ksub, p.dense, p.score, P,
-                                           hitmask + GR::s0(2) * 8);
+            build_group<W2, DSUB, NT, DBG, SCORE_T, NC>(lut + GR::lut_off(2), kSetFloats, p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
+                                                       res + GR::s0(2) * DSUB, dpad, r2 + GR::s0(2), ksub, p.dense, p.score, P,
+                                                       hitmask + GR::s0(2) * 8, IVFPQ_MAX_NSUB * 8);
         __syncthreads();
-        if (DBG && p.masks)
-            for (int i = tid; i < nsub * 8; i += NT) p.masks[(q * p.nprobe + pi) * nsub * 8 + i] = hitmask[i];
-
-        // ---- scan the cluster ----
-        const int64_t p0 = p.list_off[c];
-        const int64_t len = p.list_off[c + 1] - p0;
-        const int64_t b0 = p.list_blk[c];
-        const int64_t nblk = p.list_blk[c + 1] - b0;
-        if (nblk != (len + kPointsPerBlock - 1) / kPointsPerBlock || len < 0) {
-            if (tid == 0) atomicOr(p.status, kFlagBadList);
-            continue;
+        if (DBG && p.masks) {
+#pragma unroll
+            for (int k = 0; k < NC; ++k) {
+                const int pi = pi0 + k * p.nsplit;
+                if (pi < p.nprobe && cl[k] >= 0)
+                    for (int i = tid; i < nsub * 8; i += NT)
+                        p.masks[(q * p.nprobe + pi) * nsub * 8 + i] = hitmask[k * IVFPQ_MAX_NSUB * 8 + i];
+            }
         }
-        const unsigned char* cbase = reinterpret_cast<const unsigned char*>(p.codes_il) + b0 * GR::kBlockBytes;
-        int64_t blk = warp;   // the warp scans blocks warp, warp + kWarps, ...
+
+        // ---- scan the lists of this phase as one sequence of blocks: the warp takes blocks warp,
+        //      warp + kWarps, ...; block numbers at or beyond nblk[0] belong to the second list ----
+        const int64_t nblk_all = NC == 2 ? nblk[0] + nblk[NC - 1] : nblk[0];
+        int64_t gb = warp;
         while (true) {
             const unsigned long long tau = *tau_p;
             const uint32_t tau_hi = (uint32_t)(tau >> 32);
             bool halt = false;
-#pragma unroll 1
-            for (; blk < nblk && !halt; blk += kWarps) {
+            // one block of cluster slot K (a compile-time constant: the table bases are immediates)
+            auto scan_block = [&](auto slot_tag, int64_t blk) {
+                constexpr int K = decltype(slot_tag)::value;
                 bool stop = false;
-                const unsigned char* bp = cbase + blk * GR::kBlockBytes;
+                const unsigned char* bp = reinterpret_cast<const unsigned char*>(p.codes_il) + (b0[K] + blk) * GR::kBlockBytes;
+                const float* lutk = lut + K * kSetFloats;
+                const uint32_t* hm = hitmask + K * IVFPQ_MAX_NSUB * 8;
                 uint32_t w0[W0 >= 4 ? W0 / 4 : 1];
                 uint32_t w1[W1 >= 4 ? W1 / 4 : 1];
                 uint32_t w2[W2 >= 4 ? W2 / 4 : 1];
@@ -346,51 +403,64 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
                 unsigned long long hs = 0;
                 if constexpr (GR::kPaired) {
                     float a0 = 0.0f, a1 = 0.0f;
-                    pair_gather_words<W0 / 4, 0>(w0, pk, a0, a1);
-                    pair_gather_words<W1 / 4, 1>(w1, pk, a0, a1);
+                    pair_gather_words<W0 / 4, (int)kWin + K * kSetBytes>(w0, pk, a0, a1);
+                    pair_gather_words<W1 / 4, (int)kWin + K * kSetBytes + 128>(w1, pk, a0, a1);
                     acc = a0 + a1;
                     if (DBG) {
-                        hits_group<W0>(w0, lane, 0, hitmask, hs);
-                        hits_group<W1>(w1, lane, GR::s0(1), hitmask, hs);
+                        hits_group<W0>(w0, lane, 0, hm, hs);
+                        hits_group<W1>(w1, lane, GR::s0(1), hm, hs);
                     }
                 } else {
-                    gather_group<W0, DBG>(lut, w0, lane, 0, hitmask, acc, hs);
-                    if constexpr (W1 > 0) gather_group<W1, DBG>(lut + GR::lut_off(1), w1, lane, GR::s0(1), hitmask, acc, hs);
+                    gather_group<W0, DBG>(lutk, w0, lane, 0, hm, acc, hs);
+                    if constexpr (W1 > 0) gather_group<W1, DBG>(lutk + GR::lut_off(1), w1, lane, GR::s0(1), hm, acc, hs);
                 }
-                if constexpr (W2 > 0)
-                    gather_group<W2, DBG>(lut + GR::lut_off(2), w2, lane, GR::s0(2), hitmask, acc, hs);
+                if constexpr (W2 > 0) gather_group<W2, DBG>(lutk + GR::lut_off(2), w2, lane, GR::s0(2), hm, acc, hs);
                 const int64_t pos = blk * kPointsPerBlock + lane;
-                if (pos < len) {
+                if (pos < len[K]) {
                     if (DBG) {
-                        const int64_t vi = vprefix[pi] + pos;
+                        const int64_t vi = vprefix[pi0 + K * p.nsplit] + pos;
                         if (vi < p.visit_stride) {
                             if (p.visit_hits) p.visit_hits[q * p.visit_stride + vi] = hs;
                             if (p.visit_dist) p.visit_dist[q * p.visit_stride + vi] = acc;
-                            if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[p0 + pos];
+                            if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[p0[K] + pos];
                         }
                     }
                     if (__float_as_uint(acc) <= tau_hi) {
-                        const unsigned long long key = make_key(acc, (uint32_t)p.ids[p0 + pos]);
+                        const unsigned long long key = make_key(acc, (uint32_t)p.ids[p0[K] + pos]);
                         if (key < tau) {
                             const int slot = atomicAdd(cnt_p, 1);
-                            if (slot < kTopkCap) kbuf[slot] = key;
+                            if (slot < kCapN) kbuf[slot] = key;
                             else atomicOr(p.status, kFlagOverflow);
                             stop = slot >= kSoft;
                         }
                     }
                 }
-                halt = __any_sync(0xFFFFFFFFu, stop);
+                return __any_sync(0xFFFFFFFFu, stop);
+            };
+#pragma unroll 1
+            for (; gb < nblk_all && !halt; gb += kWarps) {
+                if (NC == 1 || gb < nblk[0]) halt = scan_block(std::integral_constant<int, 0>{}, gb);
+                else halt = scan_block(std::integral_constant<int, NC - 1>{}, gb - nblk[0]);
             }
-            // The barrier that ends the cluster (tables free for the next one).  A set flag means that a
+            // The barrier that ends the phase (tables free for the next one).  A set flag means that a
             // warp met the soft limit (it may have finished its blocks all the same): the buffer is
             // reduced to the k smallest keys and the scan resumes where it stopped.
-            if (!__syncthreads_or(blk < nblk || halt)) break;
-            topk_select<NT>(t, p.k);
+            if (!__syncthreads_or(gb < nblk_all || halt)) break;
+            topk_select<NT, CtaGroup, kCapN>(t, p.k);
         }
     }
 
-    topk_finalize<NT>(t, p.k);
-    const int n = *cnt_p;
+    // the k smallest keys, ascending
+    topk_select<NT, CtaGroup, kCapN>(t, p.k);
+    __syncthreads();
+    {
+        const int nk = min(*cnt_p, kCapN);
+        int n2 = 2;
+        while (n2 < nk) n2 <<= 1;
+        for (int i = nk + tid; i < n2; i += NT) kbuf[i] = ~0ull;
+        bitonic_sort(kbuf, n2);
+    }
+    const int n = min(*cnt_p, p.k);
     if (p.nsplit == 1) {
         for (int i = tid; i < p.k; i += NT) {
             const unsigned long long key = i < n ? kbuf[i] : kKeyPad;
@@ -403,10 +473,11 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
     }
 }
 
-template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T>
+template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T, int NC>
 cudaError_t launch_rot_inst(const ScanParams& sp, int64_t grid, int nprobe, cudaStream_t st) {
-    const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kPaired, Groups<W0, W1, W2>::kLutFloats, sp.d, nprobe, DBG);
-    auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, DBG, SCORE_T>;
+    const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kPaired, (((Groups<W0, W1, W2>::kLutFloats * 4 + 255) / 256) * 256) / 4, sp.d,
+                                       nprobe, DBG, NC);
+    auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, DBG, SCORE_T, NC>;
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<(unsigned)grid, NT, smem, st>>>(sp);
@@ -414,14 +485,14 @@ cudaError_t launch_rot_inst(const ScanParams& sp, int64_t grid, int nprobe, cuda
 }
 
 // Instances: stage dumps (score read at run time), one per score otherwise.
-template <int W0, int W1, int W2, int DSUB, int NT>
+template <int W0, int W1, int W2, int DSUB, int NT, int NC>
 cudaError_t launch_rot(const ScanParams& sp, int64_t grid, bool debug, int nprobe, cudaStream_t st) {
-    if (debug) return launch_rot_inst<W0, W1, W2, DSUB, NT, true, -1>(sp, grid, nprobe, st);
+    if (debug) return launch_rot_inst<W0, W1, W2, DSUB, NT, true, -1, NC>(sp, grid, nprobe, st);
     if (sp.score == IVFPQ_SCORE_HIT_COUNT)
-        return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_HIT_COUNT>(sp, grid, nprobe, st);
+        return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_HIT_COUNT, NC>(sp, grid, nprobe, st);
     if (sp.score == IVFPQ_SCORE_REWARD_PENALTY)
-        return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_REWARD_PENALTY>(sp, grid, nprobe, st);
-    return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_DISTANCE>(sp, grid, nprobe, st);
+        return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_REWARD_PENALTY, NC>(sp, grid, nprobe, st);
+    return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_DISTANCE, NC>(sp, grid, nprobe, st);
 }
 
 }  // namespace
@@ -450,11 +521,18 @@ bool rot_supported(int nsub, int dsub) {
 cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t grid, bool debug, int nprobe,
                             cudaStream_t st) {
     // The wide shapes run 512 threads per CTA at 64 registers, two CTAs per SM (32 warps): the table
-    // build waits on codebook loads from L2 and needs the warps to hide them.
-    if (ix->nsub == 48 && ix->dsub == 2) return launch_rot<32, 16, 0, 2, 512>(sp, grid, debug, nprobe, st);
-    if (ix->nsub == 50 && ix->dsub == 4) return launch_rot<32, 16, 2, 4, 512>(sp, grid, debug, nprobe, st);
-    if (ix->nsub == 8 && ix->dsub == 4) return launch_rot<8, 0, 0, 4, 256>(sp, grid, debug, nprobe, st);
-    if (ix->nsub == 12 && ix->dsub == 2) return launch_rot<8, 4, 0, 2, 256>(sp, grid, debug, nprobe, st);
+    // build waits on codebook loads from L2 and needs the warps to hide them.  The other arrangement
+    // (IVFPQ_ROT_KERNEL=pair when the index is loaded: 1024 threads, one CTA per SM, the tables of two
+    // probed clusters per pass over the codebook) halves the codebook traffic but measured slower
+    // (48 x 2: 4.0 -> 5.2 ms, 50 x 4: 12.1 -> 13.8 ms): one CTA's 32 warps meet at every barrier,
+    // where two independent CTAs of 16 warps overlap.
+    const bool pair = ix->rot_pair != 0;
+    if (ix->nsub == 48 && ix->dsub == 2)
+        return pair ? launch_rot<32, 16, 0, 2, 1024, 2>(sp, grid, debug, nprobe, st) : launch_rot<32, 16, 0, 2, 512, 1>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 50 && ix->dsub == 4)
+        return pair ? launch_rot<32, 16, 2, 4, 1024, 2>(sp, grid, debug, nprobe, st) : launch_rot<32, 16, 2, 4, 512, 1>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 8 && ix->dsub == 4) return launch_rot<8, 0, 0, 4, 256, 1>(sp, grid, debug, nprobe, st);
+    if (ix->nsub == 12 && ix->dsub == 2) return launch_rot<8, 4, 0, 2, 256, 1>(sp, grid, debug, nprobe, st);
     return cudaErrorNotSupported;
 }
 

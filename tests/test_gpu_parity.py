@@ -252,6 +252,41 @@ def test_16x8_kernels_forced(kernel, monkeypatch):
         lib.ivfpq_index_free(h)
 
 
+@pytest.mark.parametrize("base,kw", [("c3", {}), ("c4", {})])
+def test_wide_shapes_two_clusters_per_build_pass(base, kw, monkeypatch):
+    """48 x 2 and 50 x 4 have a second kernel arrangement (the tables of two probed clusters built in
+    one pass over the codebook), chosen when the index is loaded: top-k parity for odd and even probe
+    counts, splits, both count scores, and the stage dumps."""
+    monkeypatch.setenv("IVFPQ_ROT_KERNEL", "pair")
+    wl = Workload(small_cfg(base, n=30_000, ncomp=300, nlist=96, nq=60, chunk=16384, kmeans_iters=4, **kw))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        q = dev(wl.queries)
+        for nprobe, k, nsplit in ((7, 100, 1), (8, 1000, 1), (1, 10, 1), (9, 50, 2)):
+            lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_NSPLIT, nsplit)
+            d, i = lib.ivfpq_search_dense(h, q, nprobe, k)
+            o = oracle.search(wl.index, wl.queries, nprobe, k, dense=True)
+            check_status(h)
+            assert_topk_parity(host(d), host(i), o["dist"], o["ids"])
+            for score in (0, 1, 2):
+                d, i = lib.ivfpq_search_sparse(h, q, nprobe, dev(wl.radius_per_query), k, scale=0.9, score=score)
+                o = oracle.search(wl.index, wl.queries, nprobe, k, radius=wl.radius_per_query, scale=0.9, score=score)
+                check_status(h)
+                assert_topk_parity(host(d), host(i), o["dist"], o["ids"])
+        lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_NSPLIT, 0)
+        nq, nprobe, stride = 16, 5, 8000
+        qs, rad = wl.queries[:nq], wl.radius_per_query[:nq]
+        g = lib.ivfpq_debug_search(h, dev(qs), nprobe, 50, radius=dev(rad), scale=1.1, visit_stride=stride)
+        check_status(h)
+        g = {k2: host(v) for k2, v in g.items()}
+        o = oracle.search(wl.index, qs, nprobe, 50, radius=rad, scale=1.1, dumps=True, visit_stride=stride)
+        assert np.array_equal(g["masks"].view(np.uint32), o["masks"])
+        assert_visits_parity(g, o, wl.index.nsub)
+        assert_topk_parity(g["dist"], g["ids"], o["dist"], o["ids"])
+    finally:
+        lib.ivfpq_index_free(h)
+
+
 @pytest.mark.parametrize("kernel", ["warps16", "warps32"])
 def test_16x8_many_probes_and_splits(kernel, monkeypatch):
     """More probed clusters than the kernels stage at a time (128), alone and split over several
