@@ -396,6 +396,7 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
                 uint32_t w0[W0 >= 4 ? W0 / 4 : 1];
                 uint32_t w1[W1 >= 4 ? W1 / 4 : 1];
                 uint32_t w2[W2 >= 4 ? W2 / 4 : 1];
+                (void)lutk; (void)w1; (void)w2;   // unused in the instances without those groups
                 load_group_codes<W0>(bp, lane, w0);
                 if constexpr (W1 > 0) load_group_codes<W1>(bp + GR::chunk_off(1), lane, w1);
                 if constexpr (W2 > 0) load_group_codes<W2>(bp + GR::chunk_off(2), lane, w2);
