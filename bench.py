@@ -40,11 +40,11 @@ METRIC = "queries/sec at recall@100 (1 B200) + scan HBM GB/s as % of peak"
 UNIT = "queries/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel at the default
-# settings of a workload, from the ncu capture summarised in the named file under profiles/ (taken
-# on a smaller query batch and scaled by the points visited).  An entry is dropped (traffic: null)
-# when the kernel it describes changes.
-SCAN_DRAM_TRAFFIC = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per visited point of the dominant kernel
+# at the default settings of a workload, from the ncu capture summarised in the named file under
+# profiles/ (taken on a 1000-query batch: 7.289 GB for 475.8 M visited points; the traffic grows
+# with the points visited).  An entry is dropped (traffic: null) when the kernel it describes changes.
+SCAN_DRAM_BYTES_PER_VISIT = {"c5": (15.32, "profiles/scan16x8_1024_c5_nq1000.md")}
 
 
 def log(*a):
@@ -429,9 +429,10 @@ def run_cuda(args):
     gather_peak = props.multi_processor_count * 32 * clk * 1e6 / 1e9            # G gathers/s
     kernel = ("scan16x8_map_kernel" if map_scan else scan_kernel_name(index)) + " (selective LUT + list scan + top-k)"
     default_run = args.nq is None and args.nprobe == 0 and score == 0 and metric == 0 and not dynamic
-    traffic = SCAN_DRAM_TRAFFIC.get(args.workload) if default_run else None
+    per_visit = SCAN_DRAM_BYTES_PER_VISIT.get(args.workload) if (default_run and not map_scan) else None
+    traffic = per_visit[0] * visits if per_visit else None
     common = {"kernel": kernel, "algorithmic_bytes_per_launch": int(scan_bytes), "visits_per_launch": int(visits),
-              "kernel_ms": scan_ms, "traffic": traffic,
+              "kernel_ms": scan_ms, "traffic": traffic, "traffic_source": per_visit[1] if per_visit else None,
               "codes": f"{code_bytes_total / 1e6:.0f} MB of codes against {l2_bytes / 1e6:.0f} MB of L2"}
     if code_bytes_total > l2_bytes:
         roofline = {"bound": "hbm", "achieved": hbm_gbs, "peak": peak, "unit": "GB/s", "frac": hbm_gbs / peak,

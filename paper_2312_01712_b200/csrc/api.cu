@@ -59,7 +59,7 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     out->cbt_off = off;
     if (out->rot) off = align_up(off + (size_t)d->nsub * 256 * d->dsub * 4, 256);
     out->cnorm_off = off;
-    out->mma = (d->metric == IVFPQ_METRIC_L2 && coarse_mma_supported(d->d, d->nlist)) ? 1 : 0;
+    out->mma = coarse_mma_supported(d->d, d->nlist) ? 1 : 0;
     if (out->mma) off = align_up(off + coarse_mma_derived_bytes(d->nlist), 256);
     // entry -> points map of the sparsity-aware scan: the 16 x 8 shape under L2 (element indices are 32-bit)
     out->map = (out->rot && d->nsub == 16 && d->dsub == 8 && d->ntotal > 0 && d->ntotal * 16 < ((int64_t)1 << 32)) ? 1 : 0;

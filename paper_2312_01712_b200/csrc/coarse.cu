@@ -136,8 +136,8 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
                           float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
                           int* status, cudaStream_t st, int64_t* launches) {
     // tensor-core proposal + exact decision when the shape allows it (16-byte aligned rows)
-    const bool ip = ix->metric == IVFPQ_METRIC_IP;   // the tensor-core path and its error bound are written for L2
-    const bool mma_shape = !ip && ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
+    const bool ip = ix->metric == IVFPQ_METRIC_IP;
+    const bool mma_shape = ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
                            (reinterpret_cast<uintptr_t>(ix->cent) & 15) == 0;
     const int64_t qchunk_row = qchunk;   // queries whose full rows fit the scratch region (the plain kernels need those)
     bool mma = mma_shape, fused = false;

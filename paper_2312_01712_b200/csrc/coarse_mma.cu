@@ -150,7 +150,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1)
 coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c,
                   const float* __restrict__ cnorm, int nqc, int nlist, int kblocks, float* __restrict__ out,
                   int* __restrict__ status, int skip_last_load, int ntile_run, int out_stride,
-                  const float* __restrict__ cutp, int* __restrict__ ccount, uint2* __restrict__ cand, int ccap, int nstages) {
+                  const float* __restrict__ cutp, int* __restrict__ ccount, uint2* __restrict__ cand, int ccap, int nstages,
+                  int ip) {
+    // ip: inner-product filtering (Sec. 4.2): the values are -2 q.c, the norm term is left out.
     // ntile_run: centroid tiles to process (the first ones); out_stride: floats per row of `out`.
     // cutp != null: nothing is written to `out`; values at or under the row's cut are appended to
     // cand[q][ccount[q]++] (up to ccap entries are stored, the count keeps running).
@@ -251,7 +253,7 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         auto epi_sync = [] { asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory"); };
         if (et < kTileN) {
             const int c = blockIdx.y * kTileN + et;
-            sh->cn[0][et] = (blockIdx.y < ntile && c < nlist) ? __ldg(cnorm + c) : kInf;
+            sh->cn[0][et] = (blockIdx.y < ntile && c < nlist) ? (ip ? 0.0f : __ldg(cnorm + c)) : kInf;
         }
         epi_sync();
         // All epilogue warps meet at a named barrier once per tile, so they must leave the loop in the
@@ -263,7 +265,7 @@ coarse_mma_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             float cn_next = kInf;   // this thread's share of the next tile's norms: requested now, stored after the tile
             if (et < kTileN && ct + (int)gridDim.y < ntile) {
                 const int c = (ct + (int)gridDim.y) * kTileN + et;
-                if (c < nlist) cn_next = __ldg(cnorm + c);
+                if (c < nlist) cn_next = ip ? 0.0f : __ldg(cnorm + c);
             }
             const bool ok = mbar_wait(smem_u32(&sh->acc_full[buf]), (t >> 1) & 1, abort_word, status, limit);
             if (ok) {
@@ -372,6 +374,7 @@ __global__ void __launch_bounds__(256) cnorm_kernel(const float* __restrict__ ce
 
 // One CTA per query: cut from the approximate distances, exact re-evaluation of everything under
 // the cut, the nprobe smallest (distance, cluster id) ascending.
+template <bool IP>
 __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restrict__ approx, const float* __restrict__ queries,
                                                           const float* __restrict__ cent, const unsigned* __restrict__ cmax_bits,
                                                           int nlist, int d, int nprobe, int64_t q0,
@@ -390,7 +393,7 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
     __shared__ float red[8];
     __shared__ int ncand;
     static_assert(kQuickWords >= kTopkHistInts, "shared histogram words");
-    TopkState t{buf, &cnt, &tau, hist};
+    TopkState t{buf, &cnt, &tau, hist, IP ? kKeyPadSigned : kKeyPad};
     const int tid = threadIdx.x;
     const int64_t q = q0 + blockIdx.x;
     const float* row = approx + (size_t)blockIdx.x * nlist;
@@ -422,8 +425,18 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
     // second term covers the fp32 rounding of both sides, which grows with the number of summed
     // terms: d accumulations in the tensor-core sum and in the squared norms, d in the exact chain
     // (each at most 2^-24 of the running magnitude, itself at most |q|^2 + max|c|^2 up to a factor 2).
-    const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) +
-                      (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
+    // Inner product: the approximate cost is -q.c = half the tile value; half the TF32 term, and the
+    // rounding term on |q||c| instead of the norms.
+    const float eps = IP ? 0.625f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * sqrtf(qn) * sqrtf(cmax)
+                         : 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
+    // what the two sides are ranked by: squared distance (tile value + |q|^2, clamped at 0), or the cost -q.c
+    auto approx_of = [&](float v) { return IP ? 0.5f * v : fmaxf(v + qn, 0.0f); };
+    auto key_of = [&](float x, int id) {
+        return IP ? ((unsigned long long)ordered_bits(x) << 32) | (uint32_t)id : make_key(x, (uint32_t)id);
+    };
+    auto value_of = [&](unsigned long long key) {
+        return IP ? from_ordered_bits((uint32_t)(key >> 32)) : __uint_as_float((uint32_t)(key >> 32));
+    };
 
     // exact squared distance by the defining arithmetic (rows are 16-byte aligned, d % 4 == 0)
     auto exact = [&](int c) {
@@ -433,12 +446,19 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
             const float4 cc = __ldg(cv + j4);
             const float4 qq = *reinterpret_cast<const float4*>(qs + 4 * j4);
             float tt;
-            tt = __fsub_rn(qq.x, cc.x); a = __fmaf_rn(tt, tt, a);
-            tt = __fsub_rn(qq.y, cc.y); a = __fmaf_rn(tt, tt, a);
-            tt = __fsub_rn(qq.z, cc.z); a = __fmaf_rn(tt, tt, a);
-            tt = __fsub_rn(qq.w, cc.w); a = __fmaf_rn(tt, tt, a);
+            if (IP) {
+                a = __fmaf_rn(qq.x, cc.x, a);
+                a = __fmaf_rn(qq.y, cc.y, a);
+                a = __fmaf_rn(qq.z, cc.z, a);
+                a = __fmaf_rn(qq.w, cc.w, a);
+            } else {
+                tt = __fsub_rn(qq.x, cc.x); a = __fmaf_rn(tt, tt, a);
+                tt = __fsub_rn(qq.y, cc.y); a = __fmaf_rn(tt, tt, a);
+                tt = __fsub_rn(qq.z, cc.z); a = __fmaf_rn(tt, tt, a);
+                tt = __fsub_rn(qq.w, cc.w); a = __fmaf_rn(tt, tt, a);
+            }
         }
-        return a;
+        return IP ? -a : a;
     };
 
     bool all_exact = nprobe >= nlist || (from_list && (nlisted > ccap || nlisted < nprobe));
@@ -447,13 +467,13 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
         //      through the buffer, compacting by histogram whenever it could overflow ----
         if (nsrc <= kTopkCap) {
             // the whole row fits the buffer: every key goes to its own slot, no counting, no barriers
-            for (int c = tid; c < nsrc; c += 256) buf[c] = make_key(fmaxf(src_val(c) + qn, 0.0f), (uint32_t)src_id(c));
+            for (int c = tid; c < nsrc; c += 256) buf[c] = key_of(approx_of(src_val(c)), src_id(c));
             if (tid == 0) cnt = nsrc;
         } else {
             for (int base = 0; base < nsrc; base += 256) {
                 const int c = base + tid;
                 if (c < nsrc) {
-                    const unsigned long long key = make_key(fmaxf(src_val(c) + qn, 0.0f), (uint32_t)src_id(c));
+                    const unsigned long long key = key_of(approx_of(src_val(c)), src_id(c));
                     if (key < tau) {
                         if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
                     }
@@ -461,16 +481,17 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
                 __syncthreads();
                 const int filled = cnt;
                 __syncthreads();
-                if (filled + 256 > kTopkCap) topk_quick_compact<256>(t, nprobe, hist);
+                if (filled + 256 > kTopkCap) topk_quick_compact<256, CtaGroup, kTopkCap, IP>(t, nprobe, hist, nprobe + nprobe / 2 + 8);
             }
         }
-        topk_quick_compact<256>(t, nprobe, hist);   // starts and ends with a barrier
-        const float bound = __uint_as_float((uint32_t)(tau >> 32));   // every kept key is below it; +inf when nothing was dropped
+        // (costs of both signs span most of the bit range: their boundary bin is split again)
+        topk_quick_compact<256, CtaGroup, kTopkCap, IP>(t, nprobe, hist, nprobe + nprobe / 2 + 8);   // starts and ends with a barrier
+        const float bound = value_of(tau);   // every kept key is below it; +inf when nothing was dropped
         const float cut = bound + 2.0f * eps;
         __syncthreads();
         // ---- everything under the cut ----
         for (int c = tid; c < nsrc; c += 256) {
-            if (fmaxf(src_val(c) + qn, 0.0f) <= cut) {
+            if (approx_of(src_val(c)) <= cut) {
                 const int pos = atomicAdd(&ncand, 1);
                 if (pos < kCandCap) cand[pos] = src_id(c);
             }
@@ -484,7 +505,7 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
         for (int base = 0; base < nlist; base += 256) {
             const int c = base + tid;
             if (c < nlist) {
-                const unsigned long long key = make_key(exact(c), (uint32_t)c);
+                const unsigned long long key = key_of(exact(c), c);
                 if (key < tau) {
                     if (!topk_push(t, key)) atomicOr(status, kFlagOverflow);
                 }
@@ -493,20 +514,20 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
         }
         topk_finalize<256>(t, nprobe);
         for (int i = tid; i < nprobe; i += 256) {
-            const unsigned long long key = i < cnt ? buf[i] : kKeyPad;
+            const unsigned long long key = i < cnt ? buf[i] : t.pad;
             probe_ids[q * nprobe + i] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
-            probe_d[q * nprobe + i] = __uint_as_float((uint32_t)(key >> 32));
+            probe_d[q * nprobe + i] = value_of(key);
         }
     } else {
         const int n = ncand;   // nprobe <= n <= kCandCap = buffer size
         for (int i = tid; i < n; i += 256) {
             const int c = cand[i];
-            buf[i] = make_key(exact(c), (uint32_t)c);
+            buf[i] = key_of(exact(c), c);
         }
         __syncthreads();
         topk_emit_ranked<256>(t, n, nprobe, [&](int rank, unsigned long long key) {
             probe_ids[q * nprobe + rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
-            probe_d[q * nprobe + rank] = __uint_as_float((uint32_t)(key >> 32));
+            probe_d[q * nprobe + rank] = value_of(key);
         });
     }
 }
@@ -521,7 +542,7 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
 constexpr int kBoundPerThread = 16;
 __global__ void __launch_bounds__(256) probe_bound_kernel(const float* __restrict__ sample, int m, const float* __restrict__ queries,
                                                          const unsigned* __restrict__ cmax_bits, int d, int nprobe, int64_t q0,
-                                                         float* __restrict__ cutp, int* __restrict__ ccount) {
+                                                         float* __restrict__ cutp, int* __restrict__ ccount, int ip) {
     __shared__ int hist[256];
     __shared__ int wsum[8];
     __shared__ unsigned mm[2];
@@ -606,7 +627,9 @@ __global__ void __launch_bounds__(256) probe_bound_kernel(const float* __restric
         for (int i = 0; i < 8; ++i) qn += red[i];
         const float kth = from_ordered_bits(top);   // at or above the nprobe-th smallest sampled value
         const float cmax = __uint_as_float(*cmax_bits);
-        const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
+        // error bound of the tile value: |c|^2 - 2 q.c against the squared distance, or -2 q.c against twice the cost
+        const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) +
+                          (float)(2 * d + 8) * 5.9604645e-8f * (ip ? 2.0f * sqrtf(qn) * sqrtf(cmax) : qn + cmax);
         cutp[ql] = kth + 2.0f * eps + 1e-6f * fabsf(kth);   // the last term: the two sides add |q|^2 in different places
         ccount[ql] = 0;
     }
@@ -702,8 +725,11 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
     const float* cnorm = ix->cnorm;
     const unsigned* cmax = reinterpret_cast<const unsigned*>(reinterpret_cast<const char*>(cnorm) + align_up((size_t)ix->nlist * 4, 256));
     const size_t smem2 = (size_t)kTopkCap * 8 + (size_t)kCandCap * 4 + align_up((size_t)ix->d * 4, 16);
-    e = cudaFuncSetAttribute(probe_rerank_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    const int ip = ix->metric == IVFPQ_METRIC_IP ? 1 : 0;
+    e = ip ? cudaFuncSetAttribute(probe_rerank_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)
+           : cudaFuncSetAttribute(probe_rerank_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
     if (e != cudaSuccess) return e;
+    auto rerank = ip ? probe_rerank_kernel<true> : probe_rerank_kernel<false>;
 
     if (fused) {   // the caller checked coarse_mma_fused() and sized the scratch for it
         // scratch: [nqc][sample] values | [nqc] cuts | [nqc] counters | [nqc][kListCap] (value, cluster)
@@ -714,20 +740,20 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
         uint2* clist = reinterpret_cast<uint2*>(ccount + nqc);   // 8-byte aligned: 2 nqc words of cuts and counters before it
         const int stile = nsample / kTileN;
         coarse_mma_kernel<<<dim3(qtiles, csplit_for(stile)), kMmaThreads, smem, st>>>(
-            map_q, map_c, cnorm, nqc, ix->nlist, kblocks, sample, status, 0, stile, nsample, nullptr, nullptr, nullptr, 0, nstages);
-        probe_bound_kernel<<<nqc, 256, 0, st>>>(sample, nsample, queries, cmax, ix->d, nprobe, q0, cutp, ccount);
+            map_q, map_c, cnorm, nqc, ix->nlist, kblocks, sample, status, 0, stile, nsample, nullptr, nullptr, nullptr, 0, nstages, ip);
+        probe_bound_kernel<<<nqc, 256, 0, st>>>(sample, nsample, queries, cmax, ix->d, nprobe, q0, cutp, ccount, ip);
         coarse_mma_kernel<<<dim3(qtiles, csplit_for(ntile)), kMmaThreads, smem, st>>>(
-            map_q, map_c, cnorm, nqc, ix->nlist, kblocks, nullptr, status, 0, ntile, 0, cutp, ccount, clist, kListCap, nstages);
-        probe_rerank_kernel<<<nqc, 256, smem2, st>>>(nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
+            map_q, map_c, cnorm, nqc, ix->nlist, kblocks, nullptr, status, 0, ntile, 0, cutp, ccount, clist, kListCap, nstages, ip);
+        rerank<<<nqc, 256, smem2, st>>>(nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
                                                       probe_d, status, clist, ccount, kListCap);
         *launches += 4;
         return cudaGetLastError();
     }
     coarse_mma_kernel<<<dim3(qtiles, csplit_for(ntile)), kMmaThreads, smem, st>>>(map_q, map_c, cnorm, nqc, ix->nlist, kblocks, tile, status,
-                                                                                 ix->test_fault, ntile, ix->nlist, nullptr, nullptr, nullptr, 0, nstages);
+                                                                                 ix->test_fault, ntile, ix->nlist, nullptr, nullptr, nullptr, 0, nstages, ip);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    probe_rerank_kernel<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
+    rerank<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
                                                   probe_d, status, nullptr, nullptr, 0);
     *launches += 2;
     return cudaGetLastError();

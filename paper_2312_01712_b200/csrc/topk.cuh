@@ -373,7 +373,7 @@ __device__ inline void topk_quick_compact(const TopkState& t, int k, int* qs, in
     }
     if (tid == 0) {
         *t.cnt = 0;
-        *t.tau = bound < kKeyPad ? bound : kKeyPad;
+        *t.tau = bound < t.pad ? bound : t.pad;
     }
     G::sync();
 #pragma unroll

@@ -172,3 +172,29 @@ def test_inner_product_full_size_c4_sampled_queries():
         assert (np.diff(np.sort(gi, axis=1), axis=1) > 0).all()
     finally:
         lib.ivfpq_index_free(h)
+
+
+@pytest.mark.parametrize("nlist", [300, 1100, 8500])
+def test_inner_product_probe_lists_through_the_tensor_core_proposal(nlist):
+    """Filtering by inner product on shapes the tensor-core kernel serves (d a multiple of 4): the
+    TF32 products propose, the fused multiply-add chain decides; full rows (300, 1100 clusters) and
+    the fused epilogue lists (8500 clusters), mixed-sign inner products, centroids of very different
+    norms, duplicated centroids (ties go to the smaller cluster id)."""
+    from ivfpq_inputs import lossless_toy_index
+    rng = np.random.default_rng(nlist + 1)
+    idx, base = lossless_toy_index(seed=4, n=2 * nlist, nlist=nlist, nsub=8, dsub=8, ksub=16, spread=3.0)
+    cent = idx.coarse_centroids * rng.uniform(0.1, 30.0, (nlist, 1)).astype(F32)
+    cent[1::9] = cent[0:-1:9][: len(cent[1::9])]
+    idx.coarse_centroids = np.ascontiguousarray(cent.astype(F32))
+    idx = ip_index(idx)
+    h = lib.ivfpq_index_load(idx)
+    try:
+        q = (rng.standard_normal((130, idx.d)) * rng.uniform(0.01, 50.0, (130, 1))).astype(F32)
+        for nprobe in (1, 9, 40):
+            pid, pd = lib.ivfpq_debug_probes(h, dev(q), nprobe)
+            o = oracle.search(idx, q, nprobe, 1, dense=True, dumps=True)
+            assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
+            assert np.array_equal(host(pid), o["probe_ids"])
+            assert np.array_equal(host(pd).view(np.uint32), o["probe_d"].view(np.uint32))
+    finally:
+        lib.ivfpq_index_free(h)
