@@ -224,6 +224,12 @@ def scan_kernel_name(index) -> str:
     return "scan_rot_kernel"
 
 
+def workload_string(cfg, index, nq, nprobe, k, scale) -> str:
+    """One description of the workload for both arms."""
+    return (f"{cfg.name}: N={index.ntotal} D={index.d} nlist={index.nlist} PQ {index.nsub}x{index.dsub} (uint8 codes), "
+            f"nq={nq}/GPU, nprobe={nprobe}, k={k}, sparse search at radius scale {scale}")
+
+
 def visits_per_batch(index, probe_ids: np.ndarray) -> int:
     lens = np.diff(index.list_offsets)
     return int(lens[probe_ids].sum())
@@ -452,9 +458,7 @@ def run_cuda(args):
         "metric": METRIC, "value": nq * world * args.steps / (total_ms * 1e-3), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: N={index.ntotal} D={index.d} nlist={index.nlist} "
-                               f"PQ {index.nsub}x{index.dsub} (uint8 codes), nq={nq}/GPU, nprobe={nprobe}, k={k}, "
-                               f"sparse search at radius scale {scale}"
+        "config": {"workload": workload_string(cfg, index, nq, nprobe, k, scale)
                                + ("" if score == 0 else f", ranked by {args.score}")
                                + ("" if metric == 0 else ", inner-product similarity")
                                + ("" if not dynamic else ", query-specific thresholds (density map + regressor) computed in the step"),
@@ -556,10 +560,11 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": dt / steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{cfg.name}: N={index.ntotal} D={index.d} nlist={index.nlist} "
-                               f"PQ {index.nsub}x{index.dsub}, nprobe={nprobe}, k={k}, sparse search at radius "
-                               f"scale {scale}; each step = {sample} queries of the batch",
-                   "radius_scale": scale, "nprobe": nprobe},
+        "config": {"workload": workload_string(cfg, index, q_np.shape[0], nprobe, k, scale)
+                               + ("" if args.metric == "l2" else ", inner-product similarity"),
+                   "l2": "not applicable (host cores)", "parallelism": "1 process, OpenMP over queries",
+                   "radius_scale": scale, "nprobe": nprobe, "score": "distance", "similarity": args.metric,
+                   "reference_step": f"{sample} queries of the batch per step"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": f"{steps} steps x {sample} queries"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
