@@ -524,3 +524,47 @@ def test_full_size_c5_sampled_queries():
 
 def test_full_size_c2_sampled_queries():
     _full_size_parity("c2", 16, 128, 1.0)
+
+
+@pytest.mark.parametrize("name", ["16x8", "48x2", "50x4", "10x3"])
+def test_production_instances_equal_stage_dump_instances(shaped, name):
+    """The stage dumps come from kernel instances of their own (compiled with the dump code, score read
+    at run time, no early abandon); the instances that serve the search calls must return the same
+    top-k bit for bit, for the dense search and for every score of the sparse one."""
+    wl, h = shaped[name]
+    q = dev(wl.queries)
+    rad = dev(wl.radius_per_query)
+    for nprobe, k in ((6, 100), (11, 17)):
+        d, i = lib.ivfpq_search_dense(h, q, nprobe, k)
+        g = lib.ivfpq_debug_search(h, q, nprobe, k)
+        check_status(h)
+        assert torch.equal(i, g["ids"]) and torch.equal(d.view(torch.int32), g["dist"].view(torch.int32))
+        for score in (0, 1, 2):
+            d, i = lib.ivfpq_search_sparse(h, q, nprobe, rad, k, scale=0.9, score=score)
+            g = lib.ivfpq_debug_search(h, q, nprobe, k, radius=rad, scale=0.9, score=score)
+            check_status(h)
+            assert torch.equal(i, g["ids"]) and torch.equal(d.view(torch.int32), g["dist"].view(torch.int32))
+
+
+@pytest.mark.parametrize("kernel", ["warps16", "warps32"])
+def test_16x8_production_instances_equal_stage_dump_instances(kernel, monkeypatch):
+    """Same as above for both persistent instances of the 16 x 8 shape; the 32-warp one abandons
+    blocks early in its production form and never in its stage-dump form: same top-k bit for bit."""
+    monkeypatch.setenv("IVFPQ_SCAN_KERNEL", kernel)
+    wl = Workload(small_cfg("c1", n=40_000, ncomp=300, nlist=64, nq=70, chunk=16384, kmeans_iters=4))
+    h = lib.ivfpq_index_load(wl.index)
+    try:
+        q = dev(wl.queries)
+        lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_NSPLIT, 1)
+        for nprobe, k in ((9, 100), (30, 10)):
+            d, i = lib.ivfpq_search_dense(h, q, nprobe, k)
+            g = lib.ivfpq_debug_search(h, q, nprobe, k)
+            check_status(h)
+            assert torch.equal(i, g["ids"]) and torch.equal(d.view(torch.int32), g["dist"].view(torch.int32))
+            for score, scale in ((0, 0.6), (0, 1.0), (1, 0.8), (2, 1.2)):
+                d, i = lib.ivfpq_search_sparse(h, q, nprobe, dev(wl.radius), k, scale=scale, score=score)
+                g = lib.ivfpq_debug_search(h, q, nprobe, k, radius=dev(wl.radius), scale=scale, score=score)
+                check_status(h)
+                assert torch.equal(i, g["ids"]) and torch.equal(d.view(torch.int32), g["dist"].view(torch.int32))
+    finally:
+        lib.ivfpq_index_free(h)
