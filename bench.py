@@ -323,8 +323,14 @@ def run_cuda(args):
     def sparse_ids(s):
         return lib.ivfpq_search_sparse(h, qd, nprobe, rad_d, k, scale=s, score=score)[1].cpu().numpy()
 
-    r_dense, r1_dense, (scale, r_sparse, r1_sparse), sweep = pick_scale(sparse_ids, dense_ids, true_ids)
-    if score != 0:
+    if args.scale > 0:
+        # a fixed radius scale (an operating point of lower quality than the recall-matched one)
+        r_dense, r1_dense, (scale, r_sparse, r1_sparse), sweep = pick_scale(sparse_ids, dense_ids, true_ids, scales=(args.scale,))
+        ids = sparse_ids(args.scale)
+        scale, r_sparse, r1_sparse = args.scale, recall_at_k(ids, true_ids), recall_1_at_k(ids, true_ids)
+    else:
+        r_dense, r1_dense, (scale, r_sparse, r1_sparse), sweep = pick_scale(sparse_ids, dense_ids, true_ids)
+    if score != 0 and args.scale <= 0:
         (scale, r_sparse, r1_sparse), sweep = pick_scale_for_counts(sparse_ids, true_ids)
     assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
     log(f"[bench] recall@100 dense {r_dense:.4f}, sparse {r_sparse:.4f} at scale {scale} (sweep {sweep})")
@@ -587,6 +593,8 @@ def main():
                     help="queries timed on the CPU oracle; 0 = as many as take about 15 s (at most the batch)")
     ap.add_argument("--ref-scale", type=float, default=0.0,
                     help="radius scale of the reference arm; 0 = chosen by the CUDA arm's recall rule")
+    ap.add_argument("--scale", type=float, default=0.0,
+                    help="radius scale of the sparse search; 0 = the smallest whose recall@100 is within 0.01 of dense")
     ap.add_argument("--dynamic-radius", action="store_true",
                     help="query-specific thresholds from density maps + polynomial regressor (workload c3)")
     ap.add_argument("--metric", default="l2", choices=["l2", "ip"],
