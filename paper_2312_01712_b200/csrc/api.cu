@@ -14,7 +14,7 @@ namespace {
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 struct DerivedLayout {
-    size_t list_off_off, list_blk_off, codes_off, cbt_off, cnorm_off, chunk_first_off, map_off_off, map_pos_off, total;
+    size_t list_off_off, list_blk_off, codes_off, cbt_off, cnorm_off, blk_min_off, chunk_first_off, map_off_off, map_pos_off, total;
     int32_t map;
     int64_t nchunks;
     int32_t mma;
@@ -61,6 +61,8 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     out->cnorm_off = off;
     out->mma = coarse_mma_supported(d->d, d->nlist) ? 1 : 0;
     if (out->mma) off = align_up(off + coarse_mma_derived_bytes(d->nlist), 256);
+    out->blk_min_off = off;
+    off = align_up(off + (size_t)nblocks * 4, 256);
     // entry -> points map of the sparsity-aware scan: the 16 x 8 shape under L2 (element indices are 32-bit)
     out->map = (out->rot && d->nsub == 16 && d->dsub == 8 && d->ntotal > 0 && d->ntotal * 16 < ((int64_t)1 << 32)) ? 1 : 0;
     out->nchunks = nchunks;
@@ -249,6 +251,7 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->cbt = reinterpret_cast<const float*>(base + dl.cbt_off);
     ix->cnorm = dl.mma ? reinterpret_cast<const float*>(base + dl.cnorm_off) : nullptr;
     ix->max_list_len = dl.max_len;
+    ix->blk_min = reinterpret_cast<const uint32_t*>(base + dl.blk_min_off);
     ix->chunk_first = dl.map ? reinterpret_cast<const int32_t*>(base + dl.chunk_first_off) : nullptr;
     ix->map_off = dl.map ? reinterpret_cast<const uint32_t*>(base + dl.map_off_off) : nullptr;
     ix->map_pos = dl.map ? reinterpret_cast<const uint16_t*>(base + dl.map_pos_off) : nullptr;
@@ -297,6 +300,7 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     if (e == cudaSuccess)
         e = launch_relayout(ix, desc->codes, reinterpret_cast<uint32_t*>(base + dl.codes_off),
                             reinterpret_cast<float*>(base + dl.cbt_off), st);
+    if (e == cudaSuccess) e = launch_block_min_id(ix, reinterpret_cast<uint32_t*>(base + dl.blk_min_off), st);
     if (e == cudaSuccess) e = launch_entry_map(ix, desc->codes, st);
     if (e == cudaSuccess && ix->cnorm)
         e = launch_cnorm(ix->cent, ix->nlist, ix->d, reinterpret_cast<float*>(base + dl.cnorm_off), st);

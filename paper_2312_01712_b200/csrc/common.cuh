@@ -57,6 +57,7 @@ struct ivfpq_index {
     int32_t sparse_scan;      // IVFPQ_OPT_SPARSE_SCAN
     int32_t test_fault;       // IVFPQ_OPT_TEST_FAULT
     int64_t max_list_len;
+    const uint32_t* blk_min;     // [nblocks] smallest id (unsigned) of every 32-point block
     // host state
     int32_t device;
     int32_t sm_count;
@@ -118,6 +119,7 @@ struct WorkspaceLayout {
 WorkspaceLayout plan_workspace(const ivfpq_index* ix, int64_t nq, int32_t nprobe, int32_t k);
 
 // Launchers (return cudaError_t of the launch; count launches into *launches).
+cudaError_t launch_block_min_id(const ivfpq_index* ix, uint32_t* blk_min, cudaStream_t st);
 cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_t* codes_il, float* cbt,
                             cudaStream_t st);
 bool rot_group_widths(int nsub, int w[3]);

@@ -113,7 +113,36 @@ __global__ void __launch_bounds__(256) relayout_cbt_kernel(const float* __restri
     }
 }
 
+// Smallest id (as an unsigned number) of every 32-point block: a candidate that ties with the
+// threshold distance enters only with a smaller id than the threshold's, so a block whose smallest
+// id is not below it is decided without reading its ids (Sec. 5.3's scores tie often: hit counts
+// are small integers, and every point that missed everywhere has the same value).
+__global__ void __launch_bounds__(256) block_min_id_kernel(const int32_t* __restrict__ ids,
+                                                           const int64_t* __restrict__ list_off,
+                                                           const int64_t* __restrict__ list_blk,
+                                                           uint32_t* __restrict__ blk_min) {
+    const int list = blockIdx.x;
+    const int64_t p0 = list_off[list];
+    const int64_t len = list_off[list + 1] - p0;
+    const int64_t b0 = list_blk[list];
+    const int64_t nblk = list_blk[list + 1] - b0;
+    const int lane = threadIdx.x & 31;
+    for (int64_t b = threadIdx.x >> 5; b < nblk; b += blockDim.x >> 5) {
+        const int64_t pos = b * kPointsPerBlock + lane;
+        uint32_t v = pos < len ? (uint32_t)ids[p0 + pos] : 0xFFFFFFFFu;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+        if (lane == 0) blk_min[b0 + b] = v;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_block_min_id(const ivfpq_index* ix, uint32_t* blk_min, cudaStream_t st) {
+    if (ix->nlist > 0 && ix->nblocks > 0)
+        block_min_id_kernel<<<ix->nlist, 256, 0, st>>>(ix->ids, ix->list_off, ix->list_blk, blk_min);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_relayout(const ivfpq_index* ix, const uint8_t* codes, uint32_t* codes_il, float* cbt,
                             cudaStream_t st) {

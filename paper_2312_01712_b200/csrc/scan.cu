@@ -483,6 +483,7 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     sp.cb = ix->cb;
     sp.cbt = ix->cbt;
     sp.ids = ix->ids;
+    sp.blk_min = ix->blk_min;
     sp.codes_il = ix->codes_il;
     sp.list_off = ix->list_off;
     sp.list_blk = ix->list_blk;

@@ -59,6 +59,9 @@ constexpr uint32_t kLutWin = 0x10000;   // shared-window address of the table re
 constexpr uint32_t kCbWin = 0x20000;    // shared-window address of the shared half of the codebook (64 KB)
 constexpr int kCap = 4096;        // candidate buffer slots
 constexpr int kSoftLimit = 2048;  // compaction is requested once this many candidates are buffered
+constexpr int kAbGain = 3;        // early-abandon credit: gained per abandoned block (a completed one costs 1),
+constexpr int kAbMax = 12;        // its ceiling,
+constexpr int kAbPause = 24;      // and the blocks looked up without votes once it is used up
 constexpr int kPfDist = 3;         // blocks (per warp) that the L2 prefetch runs ahead of the scan
 static_assert(kSoftLimit + 2 * 1024 <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
 
@@ -94,7 +97,8 @@ __device__ __forceinline__ float lut_gather(uint32_t word, uint32_t pack) {
 // then some number at or above the cut.  AB = 1 tests after the second code word, AB = 2 after the
 // first and the second (the sparsity-aware search, where a miss alone can put a point out of reach).
 template <int TABLE, int AB>
-__device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[4], const uint32_t tau_cut) {
+__device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[4], const uint32_t tau_cut, bool& cut) {
+    cut = true;
     float a0 = lut_gather<0, TABLE>(cur.x, pk[0]);
     float a1 = lut_gather<1, TABLE>(cur.x, pk[0]);
     a0 += lut_gather<2, TABLE>(cur.x, pk[0]);
@@ -119,6 +123,7 @@ __device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[
     a1 += lut_gather<1, TABLE>(cur.w, pk[3]);
     a0 += lut_gather<2, TABLE>(cur.w, pk[3]);
     a1 += lut_gather<3, TABLE>(cur.w, pk[3]);
+    cut = false;
     return a0 + a1;
 }
 
@@ -250,6 +255,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
     // leaves the CTAs finishing at different times); the draw is made at the start of an item and read
     // at its end.
     for (int64_t item = blockIdx.x; item < nitems; item = *next_p) {
+        int ab_credit = kAbGain;   // per warp and query
         const int64_t q = item / p.nsplit;
         const int split = (int)(item % p.nsplit);
         const int np_item = (p.nprobe - split + p.nsplit - 1) / p.nsplit;  // probes split, split + nsplit, ...
@@ -408,14 +414,35 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                                 }
                                 // key < threshold, key = (distance, id).  The id is read only for a tie with
                                 // the threshold distance (many points can share a distance: every point
-                                // that missed in all subspaces has 16 P)
+                                // that missed in all subspaces has 16 P), and only in a block whose
+                                // smallest id is below the threshold's
                                 const uint32_t ab = __float_as_uint(acc);
-                                if (ab < tau_cut && (ab != tau_hi || (uint32_t)__ldg(p.ids + m.p0 + bpos) < tau_lo)) {
+                                if (ab < tau_cut && (ab != tau_hi || (__ldg(p.blk_min + m.b0 + (bpos >> 5)) < tau_lo &&
+                                                                      (uint32_t)__ldg(p.ids + m.p0 + bpos) < tau_lo))) {
                                     const int slot = atomicAdd(cnt_p, 1);
                                     if (slot < kCap) kbuf[slot] = make_key(acc, (uint32_t)(m.p0 + bpos));
                                     else atomicOr(p.status, kFlagOverflow);
                                     stop |= slot >= kSoftLimit;
                                 }
+                            }
+                        };
+                        // The look-ups of one block.  Early abandon pays only while blocks really are
+                        // abandoned (with small radii every point carries nearly the same sum of
+                        // penalties and none is): a warp keeps a credit that abandoned blocks raise and
+                        // completed ones lower, looks up without the votes while it is used up, and
+                        // tries again after kAbPause blocks (the threshold tightens during a scan).
+                        auto g16 = [&](const uint4 v) -> float {
+                            bool cut = false;
+                            if constexpr (AB == 0) {
+                                return gather16<TABLE, 0>(v, pk, tau_cut, cut);
+                            } else {
+                                if (ab_credit > 0) {
+                                    const float r = gather16<TABLE, AB>(v, pk, tau_cut, cut);
+                                    ab_credit = cut ? min(ab_credit + kAbGain, kAbMax) : ab_credit - 1;
+                                    return r;
+                                }
+                                ab_credit = ab_credit > -kAbPause ? ab_credit - 1 : kAbGain;
+                                return gather16<TABLE, 0>(v, pk, tau_cut, cut);
                             }
                         };
                         // Two blocks per round; each code register is refilled right after its block
@@ -427,8 +454,8 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                             if constexpr (kNT == 512) {
                                 // L2-resident lists, four warps per scheduler: the look-ups of both blocks
                                 // first (32 independent loads, four running sums), then the two tests
-                                const float acc0 = gather16<TABLE, AB>(n0, pk, tau_cut);
-                                const float acc1 = gather16<TABLE, AB>(n1, pk, tau_cut);
+                                const float acc0 = g16(n0);
+                                const float acc1 = g16(n1);
                                 if (DBG) {   // the stage dumps read the codes: keep them until then
                                     consider(n0, acc0, pos);
                                     consider(n1, acc1, pos + kWarps * kPointsPerBlock);
@@ -443,9 +470,9 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                             } else {
                                 // lists streamed from HBM: each code register is refilled as soon as its
                                 // block has been consumed
-                                consider(n0, gather16<TABLE, AB>(n0, pk, tau_cut), pos);
+                                consider(n0, g16(n0), pos);
                                 if (rem > 2) n0 = __ldg(ptr + 2 * kStep);
-                                consider(n1, gather16<TABLE, AB>(n1, pk, tau_cut), pos + kWarps * kPointsPerBlock);
+                                consider(n1, g16(n1), pos + kWarps * kPointsPerBlock);
                                 if (rem > 3) n1 = __ldg(ptr + 3 * kStep);
                             }
                             if (kPf > 0) {
@@ -458,7 +485,7 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                             halt = __any_sync(0xFFFFFFFFu, stop);
                         }
                         if (rem == 1 && !halt) {
-                            consider(n0, gather16<TABLE, AB>(n0, pk, tau_cut), pos);
+                            consider(n0, g16(n0), pos);
                             rem = 0;
                             halt = __any_sync(0xFFFFFFFFu, stop);
                         }

@@ -10,6 +10,7 @@ struct ScanParams {
     const float* cb;
     const float* cbt;
     const int32_t* ids;
+    const uint32_t* blk_min;      // smallest id of every 32-point block
     const uint32_t* codes_il;
     const int64_t* list_off;
     const int64_t* list_blk;
