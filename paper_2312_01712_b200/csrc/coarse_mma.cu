@@ -16,6 +16,8 @@
 //      answer can exceed; every centroid under the cut is re-evaluated with the defining
 //      arithmetic and the nprobe smallest (distance, cluster id) are returned.  When the cut lets
 //      too many centroids through, the CTA evaluates all of them exactly instead.
+//      Rows of at most 1024 clusters with few probes take probe_rerank_warp_kernel: the same
+//      decision with one warp per query and no block barrier.
 //
 //   Many clusters, few probes (nlist >= 8192, nprobe <= 64): the [queries][nlist] tile is never
 //   written.  A first pass runs the same kernel over the first quarter of the centroids only (at
@@ -50,6 +52,14 @@ constexpr int kTmemCols = 256;       // two accumulators of 128 columns
 constexpr unsigned kSpinLimit = 1u << 22;       // polls of one bounded wait
 constexpr unsigned kSpinLimitTest = 1u << 16;   // ... while the test-only fault option is on (about a millisecond)
 constexpr int kCandCap = kTopkCap;   // centroids that may pass the cut before the exact fallback
+constexpr int kWarpRowMax = 1024;     // clusters whose row one warp keeps in registers (probe_rerank_warp_kernel)
+constexpr int kWarpCand = 128;        // clusters under the cut that the warp kernel ranks itself
+constexpr int kWarpLowBit = 8;        // the warp kernel's bound is within 2^8 units in the last place of the order statistic
+constexpr int kWarpKernelThreads = 128;
+constexpr int kStageRow = 36;         // floats per staged slice row: 32 dimensions + padding
+__host__ __device__ inline size_t warp_rerank_smem_per_warp(int d) {
+    return align_up((size_t)d * 4, 16) + (size_t)kWarpCand * 8 + (size_t)kWarpCand * 4 + (size_t)32 * kStageRow * 4;
+}
 
 // ---- PTX wrappers -------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -442,20 +452,31 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
     auto exact = [&](int c) {
         const float4* cv = reinterpret_cast<const float4*>(cent + (size_t)c * d);
         float a = 0.0f;
-        for (int j4 = 0; j4 < (d >> 2); ++j4) {
-            const float4 cc = __ldg(cv + j4);
-            const float4 qq = *reinterpret_cast<const float4*>(qs + 4 * j4);
-            float tt;
-            if (IP) {
-                a = __fmaf_rn(qq.x, cc.x, a);
-                a = __fmaf_rn(qq.y, cc.y, a);
-                a = __fmaf_rn(qq.z, cc.z, a);
-                a = __fmaf_rn(qq.w, cc.w, a);
-            } else {
-                tt = __fsub_rn(qq.x, cc.x); a = __fmaf_rn(tt, tt, a);
-                tt = __fsub_rn(qq.y, cc.y); a = __fmaf_rn(tt, tt, a);
-                tt = __fsub_rn(qq.z, cc.z); a = __fmaf_rn(tt, tt, a);
-                tt = __fsub_rn(qq.w, cc.w); a = __fmaf_rn(tt, tt, a);
+        // one thread per centroid (the chain's order is part of the definition); its row comes from
+        // L2, so eight 16-byte loads are requested before the first is used
+        constexpr int kAhead = 8;
+        const int n4 = d >> 2;
+        for (int j0 = 0; j0 < n4; j0 += kAhead) {
+            float4 cc[kAhead];
+#pragma unroll
+            for (int u = 0; u < kAhead; ++u) cc[u] = __ldg(cv + min(j0 + u, n4 - 1));
+#pragma unroll
+            for (int u = 0; u < kAhead; ++u) {
+                if (j0 + u < n4) {
+                    const float4 qq = *reinterpret_cast<const float4*>(qs + 4 * (j0 + u));
+                    float tt;
+                    if (IP) {
+                        a = __fmaf_rn(qq.x, cc[u].x, a);
+                        a = __fmaf_rn(qq.y, cc[u].y, a);
+                        a = __fmaf_rn(qq.z, cc[u].z, a);
+                        a = __fmaf_rn(qq.w, cc[u].w, a);
+                    } else {
+                        tt = __fsub_rn(qq.x, cc[u].x); a = __fmaf_rn(tt, tt, a);
+                        tt = __fsub_rn(qq.y, cc[u].y); a = __fmaf_rn(tt, tt, a);
+                        tt = __fsub_rn(qq.z, cc[u].z); a = __fmaf_rn(tt, tt, a);
+                        tt = __fsub_rn(qq.w, cc[u].w); a = __fmaf_rn(tt, tt, a);
+                    }
+                }
             }
         }
         return IP ? -a : a;
@@ -529,6 +550,215 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
             probe_ids[q * nprobe + rank] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
             probe_d[q * nprobe + rank] = value_of(key);
         });
+    }
+}
+
+// The same decision for short rows, one warp per query: a row of at most 1024 approximate values
+// lives in the warp's registers (32 per lane, as order-preserving bits), the bound at or above the
+// nprobe-th smallest comes from a bit-by-bit search with warp-wide counts (no shared histogram, no
+// block barrier), the clusters under the cut are evaluated exactly, one per lane, and ranked by
+// counting.  32 queries are in flight per SM instead of the 4 of the CTA kernel, whose phases leave
+// most of its threads idle on such rows.  More clusters under the cut than the warp's buffer holds
+// (kWarpCand) are taken in several passes.
+template <bool IP>
+__global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kernel(
+    const float* __restrict__ approx, const float* __restrict__ queries, const float* __restrict__ cent,
+    const unsigned* __restrict__ cmax_bits, int nlist, int d, int nprobe, int64_t q0, int nqc,
+    int32_t* __restrict__ probe_ids, float* __restrict__ probe_d) {
+    extern __shared__ __align__(1024) unsigned char dyn[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int ql = blockIdx.x * (kWarpKernelThreads / 32) + warp;
+    if (ql >= nqc) return;   // whole warps; the kernel has no block barrier
+    const int64_t q = q0 + ql;
+    unsigned char* mine = dyn + (size_t)warp * warp_rerank_smem_per_warp(d);
+    float* qs = reinterpret_cast<float*>(mine);                                                   // [d]
+    unsigned long long* keys = reinterpret_cast<unsigned long long*>(mine + align_up((size_t)d * 4, 16));   // [kWarpCand]
+    int* cand = reinterpret_cast<int*>(keys + kWarpCand);                                         // [kWarpCand]
+    float* stage = reinterpret_cast<float*>(cand + kWarpCand);                                    // [32][kStageRow]
+    const float* row = approx + (size_t)ql * nlist;
+
+    // the row first: its 32 loads per lane are in flight while the query is staged
+    float rv[kWarpRowMax / 32];
+#pragma unroll
+    for (int j = 0; j < kWarpRowMax / 32; ++j) rv[j] = j * 32 + lane < nlist ? row[j * 32 + lane] : 0.0f;
+    float part = 0.0f;
+    for (int j = lane; j < d; j += 32) {
+        const float x = queries[q * d + j];
+        qs[j] = x;
+        part = fmaf(x, x, part);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
+    const float qn = part;
+    const float cmax = __uint_as_float(*cmax_bits);
+    // the error bound of probe_rerank_kernel (any order of the |q|^2 sum is covered by its second term)
+    const float eps = IP ? 0.625f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * sqrtf(qn) * sqrtf(cmax)
+                         : 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
+    __syncwarp();
+
+    // what a cluster is proposed by, as bits whose unsigned order is the order of the values:
+    // squared distance (tile value + |q|^2, clamped at 0) or the cost -q.c (half the tile value)
+    uint32_t k[kWarpRowMax / 32];
+#pragma unroll
+    for (int j = 0; j < kWarpRowMax / 32; ++j) {
+        const int c = j * 32 + lane;
+        uint32_t key = 0xFFFFFFFFu;
+        if (c < nlist) key = IP ? ordered_bits(0.5f * rv[j]) : __float_as_uint(fmaxf(rv[j] + qn, 0.0f));
+        k[j] = key;
+    }
+    // A key at or above the nprobe-th smallest: the bits that all keys share are skipped, the others
+    // are fixed from the top with warp-wide counts of the keys below a trial value, down to bit
+    // kWarpLowBit or until exactly nprobe keys lie below the trial value.
+    uint32_t lo = 0xFFFFFFFFu, hi = 0u;
+#pragma unroll
+    for (int j = 0; j < kWarpRowMax / 32; ++j) {
+        lo = min(lo, k[j]);
+        if (k[j] != 0xFFFFFFFFu) hi = max(hi, k[j]);
+    }
+    lo = __reduce_min_sync(0xFFFFFFFFu, lo);
+    hi = __reduce_max_sync(0xFFFFFFFFu, hi);
+    const int top = 31 - __clz(lo ^ hi);                       // highest bit in which two keys differ (-1: none)
+    uint32_t prefix = top >= 31 ? 0u : lo & ~((2u << max(top, 0)) - 1u) ;
+    if (top < 0) prefix = lo;
+    int unknown = top;                                          // bits unknown..0 of the order statistic are open
+    bool exact_cut = false;
+#pragma unroll 1
+    for (int b = top; b >= kWarpLowBit; --b) {
+        const uint32_t trial = prefix | (1u << b);
+        int cnt = 0;
+#pragma unroll
+        for (int j = 0; j < kWarpRowMax / 32; ++j) cnt += k[j] < trial ? 1 : 0;
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        unknown = b - 1;
+        if (cnt == nprobe) {   // exactly the wanted keys lie below the trial value
+            prefix = trial - 1u;
+            exact_cut = true;
+            break;
+        }
+        if (cnt < nprobe) prefix = trial;
+    }
+    const uint32_t bound_key = exact_cut ? prefix : (unknown >= 0 ? prefix | ((2u << unknown) - 1u) : prefix);
+    const float bound = IP ? from_ordered_bits(bound_key) : __uint_as_float(bound_key);
+    const float cut = bound + 2.0f * eps;
+
+    // ---- the clusters under the cut, in cluster order, `kWarpCand` at a time: exact values by the
+    //      defining arithmetic, then the nprobe smallest (value, cluster) so far are kept and the next
+    //      clusters join them.  Nearly always one pass.  Fewer than nprobe under the cut can only mean
+    //      that the cut is not a number: every cluster is then evaluated. ----
+    int total = 0;
+#pragma unroll
+    for (int j = 0; j < kWarpRowMax / 32; ++j) {
+        const float v = IP ? from_ordered_bits(k[j]) : __uint_as_float(k[j]);
+        const bool pass = j * 32 + lane < nlist && v <= cut;
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, pass);
+        const int pos = total + __popc(bal & ((1u << lane) - 1u));
+        if (pass && pos < kWarpCand) cand[pos] = j * 32 + lane;
+        total += __popc(bal);
+    }
+    bool all = false;
+    if (total < nprobe) {
+        all = true;
+        total = nlist;
+        for (int i = lane; i < min(nlist, kWarpCand); i += 32) cand[i] = i;
+    }
+    const int nslice = (d + 31) >> 5;
+    const int n4 = d >> 2;
+    int kept = 0, done = 0;
+    int m = min(total, kWarpCand);
+    while (true) {
+        const int cur = kept + m;
+        __syncwarp();
+        // Exact values, one cluster per lane (the order of a chain is part of the definition).  The
+        // centroid rows come from L2: 32 lanes reading 32 different rows would cost one tag look-up
+        // per lane and load, so the warp fetches slices of 32 dimensions of 32 rows with contiguous
+        // loads (8 lanes per row), passes them through shared memory (rows padded to 36 floats:
+        // conflict-free 16-byte reads), and requests the next slice before it works on the current one.
+        for (int base = kept; base < cur; base += 32) {
+            const int i = base + lane;
+            const int c = i < cur ? cand[i] : -1;
+            float a = 0.0f;
+            float4 nx[8];
+            auto request = [&](int sl) {
+    #pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int r = base + u * 4 + (lane >> 3);          // row of this lane in load u
+                    const int j4 = sl * 8 + (lane & 7);                // its 16-byte piece of the slice
+                    nx[u] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    if (r < cur && j4 < n4) nx[u] = __ldg(reinterpret_cast<const float4*>(cent + (size_t)cand[r] * d) + j4);
+                }
+            };
+            request(0);
+            for (int sl = 0; sl < nslice; ++sl) {
+                __syncwarp();   // the previous slice has been read
+    #pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    *reinterpret_cast<float4*>(stage + (u * 4 + (lane >> 3)) * kStageRow + 4 * (lane & 7)) = nx[u];
+                __syncwarp();
+                if (sl + 1 < nslice) request(sl + 1);
+                if (c >= 0) {
+    #pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int j4 = sl * 8 + u;
+                        if (j4 < n4) {
+                            const float4 cc = *reinterpret_cast<const float4*>(stage + lane * kStageRow + 4 * u);
+                            const float4 qq = *reinterpret_cast<const float4*>(qs + 4 * j4);
+                            float tt;
+                            if (IP) {
+                                a = __fmaf_rn(qq.x, cc.x, a);
+                                a = __fmaf_rn(qq.y, cc.y, a);
+                                a = __fmaf_rn(qq.z, cc.z, a);
+                                a = __fmaf_rn(qq.w, cc.w, a);
+                            } else {
+                                tt = __fsub_rn(qq.x, cc.x); a = __fmaf_rn(tt, tt, a);
+                                tt = __fsub_rn(qq.y, cc.y); a = __fmaf_rn(tt, tt, a);
+                                tt = __fsub_rn(qq.z, cc.z); a = __fmaf_rn(tt, tt, a);
+                                tt = __fsub_rn(qq.w, cc.w); a = __fmaf_rn(tt, tt, a);
+                            }
+                        }
+                    }
+                }
+            }
+            if (c >= 0) keys[i] = IP ? ((unsigned long long)ordered_bits(-a) << 32) | (uint32_t)c : make_key(a, (uint32_t)c);
+        }
+        __syncwarp();
+        done += m;
+        // ---- ranks by counting (keys are distinct: they carry the cluster) ----
+        const bool last = done >= total;
+        unsigned long long* tmp = reinterpret_cast<unsigned long long*>(stage);   // free between passes
+        for (int i = lane; i < cur; i += 32) {
+            const unsigned long long me = keys[i];
+            int rank = 0;
+            for (int j = 0; j < cur; ++j) rank += keys[j] < me ? 1 : 0;
+            if (rank < nprobe) {
+                if (last) {
+                    probe_ids[q * nprobe + rank] = (int32_t)(uint32_t)(me & 0xFFFFFFFFull);
+                    probe_d[q * nprobe + rank] = IP ? from_ordered_bits((uint32_t)(me >> 32)) : __uint_as_float((uint32_t)(me >> 32));
+                } else {
+                    tmp[rank] = me;
+                }
+            }
+        }
+        if (last) break;
+        __syncwarp();   // every rank has been counted: the nprobe smallest move to the front
+        for (int i = lane; i < nprobe; i += 32) keys[i] = tmp[i];
+        kept = nprobe;
+        // the next clusters under the cut, from the row itself (the registers that held it are in use)
+        m = min(total - done, kWarpCand - kept);
+        int run = 0;
+#pragma unroll 1
+        for (int j = 0; j < kWarpRowMax / 32; ++j) {
+            const int c = j * 32 + lane;
+            bool pass = false;
+            if (c < nlist) {
+                const float v = IP ? 0.5f * row[c] : fmaxf(row[c] + qn, 0.0f);
+                pass = all || v <= cut;
+            }
+            const unsigned bal = __ballot_sync(0xFFFFFFFFu, pass);
+            const int pos = run + __popc(bal & ((1u << lane) - 1u)) - done;
+            if (pass && pos >= 0 && pos < m) cand[kept + pos] = c;
+            run += __popc(bal);
+        }
+        __syncwarp();
     }
 }
 
@@ -753,8 +983,17 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
                                                                                  ix->test_fault, ntile, ix->nlist, nullptr, nullptr, nullptr, 0, nstages, ip);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    rerank<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
-                                                  probe_d, status, nullptr, nullptr, 0);
+    // short rows and few probes: one warp per query
+    if (ix->nlist <= kWarpRowMax && nprobe <= kWarpCand / 2 && nprobe < ix->nlist) {
+        constexpr int kWarpsPerCta = kWarpKernelThreads / 32;
+        const size_t smem3 = (size_t)kWarpsPerCta * warp_rerank_smem_per_warp(ix->d);
+        auto by_warp_kernel = ip ? probe_rerank_warp_kernel<true> : probe_rerank_warp_kernel<false>;
+        by_warp_kernel<<<(nqc + kWarpsPerCta - 1) / kWarpsPerCta, kWarpKernelThreads, smem3, st>>>(
+            tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d);
+    } else {
+        rerank<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
+                                                      probe_d, status, nullptr, nullptr, 0);
+    }
     *launches += 2;
     return cudaGetLastError();
 }

@@ -135,15 +135,15 @@ def test_probe_lists_fused_selection_large_nlist():
         lib.ivfpq_index_free(h)
 
 
-@pytest.mark.parametrize("nlist", [300, 1100, 8500])
-def test_probe_lists_large_norms_and_near_ties(nlist):
+@pytest.mark.parametrize("nlist,d", [(300, 64), (1000, 64), (1100, 64), (8500, 64), (1000, 256), (1100, 256)])
+def test_probe_lists_large_norms_and_near_ties(nlist, d):
     """Aimed at the error bound of the tensor-core proposal: coordinates around 1e4 with unit spread
     (the TF32 products are off by far more than the distances differ, so nearly every cluster falls
     under the cut), duplicated centroids (exact ties, decided by cluster id) and queries much shorter
-    than the centroids.  A loose bound would drop a true probe; the lists must stay bit-equal."""
+    than the centroids, also at the largest dimension the tensor-core path takes (256: the fp32 term of the
+    bound grows with d).  A loose bound would drop a true probe; the lists must stay bit-equal."""
     rng = np.random.default_rng(nlist)
-    d = 64
-    idx, base = lossless_toy_index(seed=9, n=2 * nlist, nlist=nlist, nsub=8, dsub=8, ksub=16, spread=1.0)
+    idx, base = lossless_toy_index(seed=9, n=2 * nlist, nlist=nlist, nsub=d // 8, dsub=8, ksub=16, spread=1.0)
     cent = (idx.coarse_centroids + 1.0e4).astype(F32)
     cent[1::7] = cent[0:-1:7][: len(cent[1::7])]           # duplicates: exact ties
     idx.coarse_centroids = cent
