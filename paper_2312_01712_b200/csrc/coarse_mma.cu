@@ -564,7 +564,11 @@ template <bool IP>
 __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kernel(
     const float* __restrict__ approx, const float* __restrict__ queries, const float* __restrict__ cent,
     const unsigned* __restrict__ cmax_bits, int nlist, int d, int nprobe, int64_t q0, int nqc,
-    int32_t* __restrict__ probe_ids, float* __restrict__ probe_d) {
+    int32_t* __restrict__ probe_ids, float* __restrict__ probe_d, const uint2* __restrict__ clist,
+    const int* __restrict__ ccount, int ccap) {
+    // clist != null: the proposals are the (value, cluster) pairs the filtering epilogue kept for the
+    // query (at most ccap <= kWarpRowMax); a list that did not fit, or is shorter than nprobe, means:
+    // every cluster is evaluated exactly
     extern __shared__ __align__(1024) unsigned char dyn[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int ql = blockIdx.x * (kWarpKernelThreads / 32) + warp;
@@ -576,11 +580,17 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kerne
     int* cand = reinterpret_cast<int*>(keys + kWarpCand);                                         // [kWarpCand]
     float* stage = reinterpret_cast<float*>(cand + kWarpCand);                                    // [32][kStageRow]
     const float* row = approx + (size_t)ql * nlist;
+    const bool from_list = clist != nullptr;
+    const uint2* cl = clist + (size_t)ql * ccap;
+    const int nlisted = from_list ? ccount[ql] : 0;
+    const int nsrc = from_list ? min(nlisted, ccap) : nlist;
+    auto src_val = [&](int i) { return from_list ? __uint_as_float(cl[i].x) : row[i]; };
+    auto src_id = [&](int i) { return from_list ? (int)cl[i].y : i; };
 
     // the row first: its 32 loads per lane are in flight while the query is staged
     float rv[kWarpRowMax / 32];
 #pragma unroll
-    for (int j = 0; j < kWarpRowMax / 32; ++j) rv[j] = j * 32 + lane < nlist ? row[j * 32 + lane] : 0.0f;
+    for (int j = 0; j < kWarpRowMax / 32; ++j) rv[j] = j * 32 + lane < nsrc ? src_val(j * 32 + lane) : 0.0f;
     float part = 0.0f;
     for (int j = lane; j < d; j += 32) {
         const float x = queries[q * d + j];
@@ -603,7 +613,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kerne
     for (int j = 0; j < kWarpRowMax / 32; ++j) {
         const int c = j * 32 + lane;
         uint32_t key = 0xFFFFFFFFu;
-        if (c < nlist) key = IP ? ordered_bits(0.5f * rv[j]) : __float_as_uint(fmaxf(rv[j] + qn, 0.0f));
+        if (c < nsrc) key = IP ? ordered_bits(0.5f * rv[j]) : __float_as_uint(fmaxf(rv[j] + qn, 0.0f));
         k[j] = key;
     }
     // A key at or above the nprobe-th smallest: the bits that all keys share are skipped, the others
@@ -649,14 +659,15 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kerne
 #pragma unroll
     for (int j = 0; j < kWarpRowMax / 32; ++j) {
         const float v = IP ? from_ordered_bits(k[j]) : __uint_as_float(k[j]);
-        const bool pass = j * 32 + lane < nlist && v <= cut;
+        const bool pass = j * 32 + lane < nsrc && v <= cut;
         const unsigned bal = __ballot_sync(0xFFFFFFFFu, pass);
         const int pos = total + __popc(bal & ((1u << lane) - 1u));
-        if (pass && pos < kWarpCand) cand[pos] = j * 32 + lane;
+        if (pass && pos < kWarpCand) cand[pos] = src_id(j * 32 + lane);
         total += __popc(bal);
     }
     bool all = false;
-    if (total < nprobe) {
+    if (total < nprobe || (from_list && nlisted > ccap)) {
+        __syncwarp();
         all = true;
         total = nlist;
         for (int i = lane; i < min(nlist, kWarpCand); i += 32) cand[i] = i;
@@ -744,19 +755,23 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kerne
         kept = nprobe;
         // the next clusters under the cut, from the row itself (the registers that held it are in use)
         m = min(total - done, kWarpCand - kept);
-        int run = 0;
+        if (all) {
+            for (int i = lane; i < m; i += 32) cand[kept + i] = done + i;
+        } else {
+            int run = 0;
 #pragma unroll 1
-        for (int j = 0; j < kWarpRowMax / 32; ++j) {
-            const int c = j * 32 + lane;
-            bool pass = false;
-            if (c < nlist) {
-                const float v = IP ? 0.5f * row[c] : fmaxf(row[c] + qn, 0.0f);
-                pass = all || v <= cut;
+            for (int j = 0; j < kWarpRowMax / 32; ++j) {
+                const int i = j * 32 + lane;
+                bool pass = false;
+                if (i < nsrc) {
+                    const float v = IP ? 0.5f * src_val(i) : fmaxf(src_val(i) + qn, 0.0f);
+                    pass = v <= cut;
+                }
+                const unsigned bal = __ballot_sync(0xFFFFFFFFu, pass);
+                const int pos = run + __popc(bal & ((1u << lane) - 1u)) - done;
+                if (pass && pos >= 0 && pos < m) cand[kept + pos] = src_id(i);
+                run += __popc(bal);
             }
-            const unsigned bal = __ballot_sync(0xFFFFFFFFu, pass);
-            const int pos = run + __popc(bal & ((1u << lane) - 1u)) - done;
-            if (pass && pos >= 0 && pos < m) cand[kept + pos] = c;
-            run += __popc(bal);
         }
         __syncwarp();
     }
@@ -974,8 +989,16 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
         probe_bound_kernel<<<nqc, 256, 0, st>>>(sample, nsample, queries, cmax, ix->d, nprobe, q0, cutp, ccount, ip);
         coarse_mma_kernel<<<dim3(qtiles, csplit_for(ntile)), kMmaThreads, smem, st>>>(
             map_q, map_c, cnorm, nqc, ix->nlist, kblocks, nullptr, status, 0, ntile, 0, cutp, ccount, clist, kListCap, nstages, ip);
-        rerank<<<nqc, 256, smem2, st>>>(nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
-                                                      probe_d, status, clist, ccount, kListCap);
+        if (nprobe <= kWarpCand / 2 && nprobe < ix->nlist && kListCap <= kWarpRowMax) {
+            constexpr int kWarpsPerCta = kWarpKernelThreads / 32;
+            const size_t smem3 = (size_t)kWarpsPerCta * warp_rerank_smem_per_warp(ix->d);
+            auto by_warp_kernel = ip ? probe_rerank_warp_kernel<true> : probe_rerank_warp_kernel<false>;
+            by_warp_kernel<<<(nqc + kWarpsPerCta - 1) / kWarpsPerCta, kWarpKernelThreads, smem3, st>>>(
+                nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d, clist, ccount, kListCap);
+        } else {
+            rerank<<<nqc, 256, smem2, st>>>(nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
+                                                          probe_d, status, clist, ccount, kListCap);
+        }
         *launches += 4;
         return cudaGetLastError();
     }
@@ -989,7 +1012,7 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
         const size_t smem3 = (size_t)kWarpsPerCta * warp_rerank_smem_per_warp(ix->d);
         auto by_warp_kernel = ip ? probe_rerank_warp_kernel<true> : probe_rerank_warp_kernel<false>;
         by_warp_kernel<<<(nqc + kWarpsPerCta - 1) / kWarpsPerCta, kWarpKernelThreads, smem3, st>>>(
-            tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d);
+            tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d, nullptr, nullptr, 0);
     } else {
         rerank<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
                                                       probe_d, status, nullptr, nullptr, 0);
