@@ -59,9 +59,6 @@ constexpr uint32_t kLutWin = 0x10000;   // shared-window address of the table re
 constexpr uint32_t kCbWin = 0x20000;    // shared-window address of the shared half of the codebook (64 KB)
 constexpr int kCap = 4096;        // candidate buffer slots
 constexpr int kSoftLimit = 2048;  // compaction is requested once this many candidates are buffered
-constexpr int kAbGain = 3;        // early-abandon credit: gained per abandoned block (a completed one costs 1),
-constexpr int kAbMax = 12;        // its ceiling,
-constexpr int kAbPause = 24;      // and the blocks looked up without votes once it is used up
 constexpr int kPfDist = 3;         // blocks (per warp) that the L2 prefetch runs ahead of the scan
 static_assert(kSoftLimit + 2 * 1024 <= kCap && IVFPQ_MAX_K < kSoftLimit, "candidate buffer limits");
 
@@ -97,8 +94,7 @@ __device__ __forceinline__ float lut_gather(uint32_t word, uint32_t pack) {
 // then some number at or above the cut.  AB = 1 tests after the second code word, AB = 2 after the
 // first and the second (the sparsity-aware search, where a miss alone can put a point out of reach).
 template <int TABLE, int AB>
-__device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[4], const uint32_t tau_cut, bool& cut) {
-    cut = true;
+__device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[4], const uint32_t tau_cut) {
     float a0 = lut_gather<0, TABLE>(cur.x, pk[0]);
     float a1 = lut_gather<1, TABLE>(cur.x, pk[0]);
     a0 += lut_gather<2, TABLE>(cur.x, pk[0]);
@@ -123,7 +119,6 @@ __device__ __forceinline__ float gather16(const uint4 cur, const uint32_t (&pk)[
     a1 += lut_gather<1, TABLE>(cur.w, pk[3]);
     a0 += lut_gather<2, TABLE>(cur.w, pk[3]);
     a1 += lut_gather<3, TABLE>(cur.w, pk[3]);
-    cut = false;
     return a0 + a1;
 }
 
@@ -255,7 +250,6 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
     // leaves the CTAs finishing at different times); the draw is made at the start of an item and read
     // at its end.
     for (int64_t item = blockIdx.x; item < nitems; item = *next_p) {
-        int ab_credit = kAbGain;   // per warp and query
         const int64_t q = item / p.nsplit;
         const int split = (int)(item % p.nsplit);
         const int np_item = (p.nprobe - split + p.nsplit - 1) / p.nsplit;  // probes split, split + nsplit, ...
@@ -426,25 +420,8 @@ __global__ void __launch_bounds__(NT, 1) scan16x8_kernel(const ScanParams p, con
                                 }
                             }
                         };
-                        // The look-ups of one block.  Early abandon pays only while blocks really are
-                        // abandoned (with small radii every point carries nearly the same sum of
-                        // penalties and none is): a warp keeps a credit that abandoned blocks raise and
-                        // completed ones lower, looks up without the votes while it is used up, and
-                        // tries again after kAbPause blocks (the threshold tightens during a scan).
-                        auto g16 = [&](const uint4 v) -> float {
-                            bool cut = false;
-                            if constexpr (AB == 0) {
-                                return gather16<TABLE, 0>(v, pk, tau_cut, cut);
-                            } else {
-                                if (ab_credit > 0) {
-                                    const float r = gather16<TABLE, AB>(v, pk, tau_cut, cut);
-                                    ab_credit = cut ? min(ab_credit + kAbGain, kAbMax) : ab_credit - 1;
-                                    return r;
-                                }
-                                ab_credit = ab_credit > -kAbPause ? ab_credit - 1 : kAbGain;
-                                return gather16<TABLE, 0>(v, pk, tau_cut, cut);
-                            }
-                        };
+                        // the look-ups of one block
+                        auto g16 = [&](const uint4 v) -> float { return gather16<TABLE, AB>(v, pk, tau_cut); };
                         // Two blocks per round; each code register is refilled right after its block
                         // has been consumed (no copies).  The fill level of the candidate buffer is
                         // only looked at by lanes that push: a warp leaves the loop at the end of a
@@ -536,7 +513,9 @@ template <int NT>
 cudaError_t launch_nt(const ScanParams& sp, int64_t grid, int64_t nitems, bool debug, cudaStream_t st) {
     constexpr int kAbDense = NT == 1024 ? 1 : 0, kAbSparse = NT == 1024 ? 2 : 0;
     if (debug) return launch_inst<NT, true, -1, 0>(sp, grid, nitems, st);
-    if (sp.score == IVFPQ_SCORE_HIT_COUNT) return launch_inst<NT, false, IVFPQ_SCORE_HIT_COUNT, kAbSparse>(sp, grid, nitems, st);
+    // (at the radii where the hit count ranks best nearly every point misses nearly everywhere: the
+    // threshold stays above the misses of half the subspaces, no block is abandoned: no votes)
+    if (sp.score == IVFPQ_SCORE_HIT_COUNT) return launch_inst<NT, false, IVFPQ_SCORE_HIT_COUNT, 0>(sp, grid, nitems, st);
     if (sp.score == IVFPQ_SCORE_REWARD_PENALTY) return launch_inst<NT, false, IVFPQ_SCORE_REWARD_PENALTY, kAbSparse>(sp, grid, nitems, st);
     if (sp.dense) return launch_inst<NT, false, IVFPQ_SCORE_DISTANCE, kAbDense>(sp, grid, nitems, st);
     return launch_inst<NT, false, IVFPQ_SCORE_DISTANCE, kAbSparse>(sp, grid, nitems, st);
