@@ -215,8 +215,9 @@ SCORE_NAMES = {"distance": 0, "hit_count": 1, "reward_penalty": 2}
 
 def scan_kernel_name(index) -> str:
     """Name of the kernel the library picks for this index (same rule as ivfpq_index_load)."""
+    rot_shapes = {(16, 8), (48, 2), (50, 4), (8, 4), (12, 2)}
     if getattr(index, "metric", 0) == 1:
-        return "scan_ip_kernel"
+        return "scan_rot_kernel<inner product>" if (index.nsub, index.dsub) in rot_shapes else "scan_ip_kernel"
     if (index.nsub, index.dsub) == (16, 8):
         forced = os.environ.get("IVFPQ_SCAN_KERNEL")
         wide = forced == "warps32" or (forced != "warps16" and index.ntotal // index.nlist >= 2048)

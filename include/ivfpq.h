@@ -31,9 +31,10 @@
  *       id) per query, padded with (-inf, -1).
  *   out_dist, probe_d and the dumps then hold similarities.  Defining arithmetic: inner products
  *   and |e|^2 as one fused multiply-add per dimension, ascending; |q_s - e|^2 as for L2; the test
- *   compares with the fp32 sum R^2 + |e|^2.  The count scores, ivfpq_probe_static and the
- *   specialised scan kernels are L2-only: an inner-product index is served by the generic scan
- *   kernel (its filtering goes through the same tensor-core proposal + exact decision as L2).
+ *   compares with the fp32 sum R^2 + |e|^2.  The count scores, ivfpq_probe_static, the entry ->
+ *   points map and the persistent 16 x 8 kernels are L2-only; an inner-product index of a shape
+ *   with a conflict-free code layout is served by that layout's scan kernel, other shapes by the
+ *   generic one (filtering goes through the same tensor-core proposal + exact decision as L2).
  *
  * Conventions for every entry point:
  *   - returns IVFPQ_OK (0) or a negative IVFPQ_ERR_* code; never throws, never aborts;

@@ -52,8 +52,7 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     out->list_blk_off = off;
     off = align_up(off + sizeof(int64_t) * (size_t)(d->nlist + 1), 256);
     out->codes_off = off;
-    // the rotated layouts belong to the L2-only kernels
-    out->rot = (d->metric == IVFPQ_METRIC_L2 && rot_supported(d->nsub, d->dsub) && rot_group_widths(d->nsub, out->gw)) ? 1 : 0;
+    out->rot = (rot_supported(d->nsub, d->dsub) && rot_group_widths(d->nsub, out->gw)) ? 1 : 0;
     out->block_bytes = out->rot ? rot_block_bytes(out->gw) : kPointsPerBlock * out->nw * 4;
     off = align_up(off + (size_t)nblocks * out->block_bytes, 256);
     out->cbt_off = off;
@@ -64,7 +63,7 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     out->blk_min_off = off;
     off = align_up(off + (size_t)nblocks * 4, 256);
     // entry -> points map of the sparsity-aware scan: the 16 x 8 shape under L2 (element indices are 32-bit)
-    out->map = (out->rot && d->nsub == 16 && d->dsub == 8 && d->ntotal > 0 && d->ntotal * 16 < ((int64_t)1 << 32)) ? 1 : 0;
+    out->map = (out->rot && d->metric == IVFPQ_METRIC_L2 && d->nsub == 16 && d->dsub == 8 && d->ntotal > 0 && d->ntotal * 16 < ((int64_t)1 << 32)) ? 1 : 0;
     out->nchunks = nchunks;
     out->chunk_first_off = out->map_off_off = out->map_pos_off = off;
     if (out->map) {

@@ -526,7 +526,9 @@ cudaError_t launch_scan(const SearchArgs& a, const WorkspaceLayout& wl, char* ws
     const int64_t grid = a.nq * sp.nsplit;
     cudaError_t e;
     const bool ip = ix->metric == IVFPQ_METRIC_IP;
-    if (ip)
+    if (ip && ix->rot)
+        e = launch_scan_rot(ix, sp, grid, a.debug, a.nprobe, st);
+    else if (ip)
         e = a.debug ? launch_ip<true>(sp, grid, smem, st) : launch_ip<false>(sp, grid, smem, st);
     else if (pers_shape(ix) && use_entry_map(ix, a))
         e = launch_scan16x8_map(ix, sp, grid, a.debug, a.nprobe, st);

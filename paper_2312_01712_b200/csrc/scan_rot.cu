@@ -73,10 +73,19 @@ __host__ __device__ inline size_t rot_aux_bytes(int d, int nc) {
 
 // Dynamic shared memory of a launch.  Paired layout: everything up to the fixed table address
 // (whatever the window offset of the allocation turns out to be), the tables, the debug area.
-__host__ __device__ inline size_t rot_smem_bytes(bool paired, int lut_floats, int d, int nprobe, bool dbg, int nc) {
+// Inner product: the lists of a tile of probed clusters are scanned as one sequence of blocks.
+constexpr int kIpTile = 64;
+struct IpProbe {
+    long long p0, b0;   // first point and first block of the list
+    int len, blk_end;   // points of the list; blocks of the tile up to and including this list
+    float base;         // -(q.c)
+    int pi;             // probe number, -1: invalid cluster id
+};
+__host__ __device__ inline size_t rot_smem_bytes(bool paired, int lut_floats, int d, int nprobe, bool dbg, int nc, bool ip = false) {
     size_t b = paired ? (size_t)pair_win(nc) : rot_aux_bytes(d, nc);
     b += (size_t)nc * lut_floats * 4;
-    if (dbg) b += (size_t)nc * IVFPQ_MAX_NSUB * 8 * 4 + (size_t)(nprobe + 1) * 8;
+    if (dbg) b += (size_t)nc * IVFPQ_MAX_NSUB * 8 * 4 + align_up((size_t)(nprobe + 1) * 8, 16);
+    if (ip) b += (size_t)kIpTile * sizeof(IpProbe);
     return b;
 }
 
@@ -85,7 +94,9 @@ __host__ __device__ inline size_t rot_smem_bytes(bool paired, int lut_floats, in
 // and measured against the residuals of all NC clusters (the codebook comes through L2: with two
 // clusters per pass its traffic per table halves).  lut_step / res_step / hm_step: distance between
 // the clusters' tables, residuals and stage-dump masks.
-template <int W, int DSUB, int NT, bool DBG, int SCORE_T, int NC, int RS = row_stride(W)>
+// IP (inner-product index, paper Sec. 4.2): `res_g` is the query itself; an entry is selected when
+// |q_s - e|^2 <= R_s^2 + |e|^2 and its slot then holds -(q_s.e), the miss constant otherwise.
+template <int W, int DSUB, int NT, bool DBG, int SCORE_T, int NC, int RS = row_stride(W), bool IP = false>
 __device__ __forceinline__ void build_group(float* __restrict__ lutg, int lut_step, const float* __restrict__ cbt_g,
                                             const float* __restrict__ res_g, int res_step, const float* __restrict__ r2_g,
                                             int ksub, bool dense, int score, float P, uint32_t* hitmask_g, int hm_step) {
@@ -131,17 +142,27 @@ __device__ __forceinline__ void build_group(float* __restrict__ lutg, int lut_st
             }
 #pragma unroll
             for (int k = 0; k < NC; ++k) {
+                float en2 = 0.0f, ipv = 0.0f;
 #pragma unroll
                 for (int j = 0; j < DSUB; ++j) {
                     const float tt = __fsub_rn(r[k][j], ev[j]);
                     d2[k] = __fmaf_rn(tt, tt, d2[k]);
+                    if (IP) {
+                        en2 = __fmaf_rn(ev[j], ev[j], en2);
+                        ipv = __fmaf_rn(r[k][j], ev[j], ipv);
+                    }
                 }
-                hit[k] = dense || d2[k] <= thr;
+                if (IP) {
+                    hit[k] = dense || d2[k] <= __fadd_rn(thr, en2);
+                    d2[k] = -ipv;
+                } else {
+                    hit[k] = dense || d2[k] <= thr;
+                }
             }
         }
 #pragma unroll
         for (int k = 0; k < NC; ++k) {
-            const float val = table_value<SCORE_T>(score, hit[k], d2[k], thr, P);
+            const float val = IP ? (hit[k] ? d2[k] : P) : table_value<SCORE_T>(score, hit[k], d2[k], thr, P);
             float* row = lutg + k * lut_step + e * RS + c;
 #pragma unroll
             for (int it = 0; it < NCOPY; ++it) {
@@ -232,8 +253,13 @@ __device__ __forceinline__ void load_group_codes(const unsigned char* __restrict
 // NC = clusters per phase: 1 (one table at a time) or 2 (1024 threads, one CTA per SM; the tables of
 // two probed clusters are built in one pass over the codebook, then both lists are scanned as one
 // sequence of blocks).
-template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T, int NC>
+// IP: the inner-product index.  One table per query (built from the query, before the first
+// cluster) serves all its probed clusters; a point's cost is -(q.c) from the filtering stage plus one
+// slot per subspace; keys carry the cost under the order-preserving bit map (costs can be negative)
+// and the reported value is the similarity, -cost.
+template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T, int NC, bool IP = false>
 __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const ScanParams p) {
+    static_assert(!IP || NC == 1, "the inner-product instance works on one cluster at a time");
     using GR = Groups<W0, W1, W2>;
     constexpr int kWarps = NT / 32;
     constexpr int kCapN = cand_cap(NC);
@@ -273,6 +299,8 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
     float* lut = reinterpret_cast<float*>(smem + lut_at);                                           // [NC] sets of kSetBytes
     uint32_t* hitmask = reinterpret_cast<uint32_t*>(smem + lut_at + (size_t)NC * kSetBytes);       // DBG only: [NC][64][8]
     long long* vprefix = reinterpret_cast<long long*>(hitmask + NC * IVFPQ_MAX_NSUB * 8);           // DBG only
+    IpProbe* ipm = reinterpret_cast<IpProbe*>(smem + lut_at + (size_t)NC * kSetBytes +
+                                              (DBG ? (size_t)NC * IVFPQ_MAX_NSUB * 8 * 4 + align_up((size_t)(p.nprobe + 1) * 8, 16) : 0));   // IP only
     constexpr int kSetFloats = kSetBytes / 4;
     // paired layout: column offsets (lane ^ i) * 4 of the 32 steps, four per register
     uint32_t pk[GR::kPaired ? 8 : 1];
@@ -288,7 +316,7 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
 
     const int64_t q = blockIdx.x / p.nsplit;
     const int split = blockIdx.x % p.nsplit;
-    TopkState t{kbuf, cnt_p, tau_p, hist_p};
+    TopkState t{kbuf, cnt_p, tau_p, hist_p, IP ? kKeyPadSigned : kKeyPad};
 
     if (tid < nsub) {
         float v = 0.0f;
@@ -319,6 +347,157 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
         }
     }
 
+    // the tables of all groups from the vector(s) in `res`
+    auto build_tables = [&]() {
+        build_group<W0, DSUB, NT, DBG, SCORE_T, NC, GR::stride(0), IP>(lut, kSetFloats, p.cbt, res, dpad, r2, ksub, p.dense, p.score, P,
+                                                                  hitmask, IVFPQ_MAX_NSUB * 8);
+        if constexpr (W1 > 0)
+            build_group<W1, DSUB, NT, DBG, SCORE_T, NC, GR::stride(1), IP>(lut + GR::lut_off(1), kSetFloats,
+                                                                      p.cbt + (size_t)GR::s0(1) * 256 * DSUB, res + GR::s0(1) * DSUB, dpad,
+                                                                      r2 + GR::s0(1), ksub, p.dense, p.score, P,
+                                                                      hitmask + GR::s0(1) * 8, IVFPQ_MAX_NSUB * 8);
+        if constexpr (W2 > 0)
+            build_group<W2, DSUB, NT, DBG, SCORE_T, NC, row_stride(W2), IP>(lut + GR::lut_off(2), kSetFloats, p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
+                                                       res + GR::s0(2) * DSUB, dpad, r2 + GR::s0(2), ksub, p.dense, p.score, P,
+                                                       hitmask + GR::s0(2) * 8, IVFPQ_MAX_NSUB * 8);
+    };
+    if (IP) {
+        for (int j = tid; j < d; j += NT) res[j] = p.queries[q * d + j];
+        if (DBG)
+            for (int i = tid; i < NC * IVFPQ_MAX_NSUB * 8; i += NT) hitmask[i] = 0;
+        __syncthreads();
+        build_tables();
+        __syncthreads();
+    }
+
+    // One block of 32 points of the list that starts at block B0 / point P0 and holds LEN points, against the
+    // tables of cluster slot K (a compile-time constant: the table bases are immediates); PI = its probe
+    // number (stage dumps), BASE = -(q.c) (inner product).  Returns whether the warp has to stop.
+    auto scan_block = [&](auto slot_tag, int64_t blk, int64_t B0, int64_t LEN, int64_t P0, int PI, float BASE,
+                  unsigned long long tau, uint32_t tau_hi) -> bool {
+        constexpr int K = decltype(slot_tag)::value;
+        bool stop = false;
+        const unsigned char* bp = reinterpret_cast<const unsigned char*>(p.codes_il) + (B0 + blk) * GR::kBlockBytes;
+        const float* lutk = lut + K * kSetFloats;
+        const uint32_t* hm = hitmask + K * IVFPQ_MAX_NSUB * 8;
+        uint32_t w0[W0 >= 4 ? W0 / 4 : 1];
+        uint32_t w1[W1 >= 4 ? W1 / 4 : 1];
+        uint32_t w2[W2 >= 4 ? W2 / 4 : 1];
+        (void)lutk; (void)w1; (void)w2;   // unused in the instances without those groups
+        load_group_codes<W0>(bp, lane, w0);
+        if constexpr (W1 > 0) load_group_codes<W1>(bp + GR::chunk_off(1), lane, w1);
+        if constexpr (W2 > 0) load_group_codes<W2>(bp + GR::chunk_off(2), lane, w2);
+        float acc = 0.0f;
+        unsigned long long hs = 0;
+        if constexpr (GR::kPaired) {
+            float a0 = 0.0f, a1 = 0.0f;
+            pair_gather_words<W0 / 4, (int)kWin + K * kSetBytes>(w0, pk, a0, a1);
+            pair_gather_words<W1 / 4, (int)kWin + K * kSetBytes + 128>(w1, pk, a0, a1);
+            acc = a0 + a1;
+            if (DBG) {
+                hits_group<W0>(w0, lane, 0, hm, hs);
+                hits_group<W1>(w1, lane, GR::s0(1), hm, hs);
+            }
+        } else {
+            gather_group<W0, DBG>(lutk, w0, lane, 0, hm, acc, hs);
+            if constexpr (W1 > 0) gather_group<W1, DBG>(lutk + GR::lut_off(1), w1, lane, GR::s0(1), hm, acc, hs);
+        }
+        if constexpr (W2 > 0) gather_group<W2, DBG>(lutk + GR::lut_off(2), w2, lane, GR::s0(2), hm, acc, hs);
+        if (IP) acc += BASE;
+        const int64_t pos = blk * kPointsPerBlock + lane;
+        if (pos < LEN) {
+            if (DBG) {
+                const int64_t vi = vprefix[PI] + pos;
+                if (vi < p.visit_stride) {
+                    if (p.visit_hits) p.visit_hits[q * p.visit_stride + vi] = hs;
+                    if (p.visit_dist) p.visit_dist[q * p.visit_stride + vi] = IP ? -acc : acc;
+                    if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[P0 + pos];
+                }
+            }
+            const uint32_t ab = IP ? ordered_bits(acc) : __float_as_uint(acc);
+            if (ab <= tau_hi) {
+                const unsigned long long key = ((unsigned long long)ab << 32) | (uint32_t)p.ids[P0 + pos];
+                if (key < tau) {
+                    const int slot = atomicAdd(cnt_p, 1);
+                    if (slot < kCapN) kbuf[slot] = key;
+                    else atomicOr(p.status, kFlagOverflow);
+                    stop = slot >= kSoft;
+                }
+            }
+        }
+        return __any_sync(0xFFFFFFFFu, stop);
+    };
+
+    // ---- inner product: the table is the same for every cluster, so nothing separates the lists: a
+    //      tile of up to kIpTile probed clusters is staged (one thread per cluster: the chain of
+    //      dependent loads from the probe list to the list tables is paid once per tile, not once per
+    //      cluster) and its lists are scanned as one sequence of blocks, with a barrier only when the
+    //      candidate buffer has to be reduced ----
+    if constexpr (IP) {
+        const int np_item = (p.nprobe - split + p.nsplit - 1) / p.nsplit;   // probes split, split + nsplit, ...
+        for (int t0 = 0; t0 < np_item; t0 += kIpTile) {
+            const int nt = min(kIpTile, np_item - t0);
+            __syncthreads();   // the previous tile's entries are no longer read
+            if (tid < nt) {
+                IpProbe m;
+                m.pi = split + (t0 + tid) * p.nsplit;
+                m.p0 = m.b0 = 0;
+                m.len = m.blk_end = 0;
+                m.base = 0.0f;
+                const int c = p.probe_ids[q * p.nprobe + m.pi];
+                if (c < 0 || c >= p.nlist) {
+                    atomicOr(p.status, kFlagBadList);
+                    m.pi = -1;
+                } else {
+                    m.p0 = p.list_off[c];
+                    const int64_t len = p.list_off[c + 1] - m.p0;
+                    m.b0 = p.list_blk[c];
+                    const int64_t nblk = p.list_blk[c + 1] - m.b0;
+                    if (nblk != (len + kPointsPerBlock - 1) / kPointsPerBlock || len < 0) {
+                        atomicOr(p.status, kFlagBadList);
+                    } else {
+                        m.len = (int)len;
+                        m.blk_end = (int)nblk;
+                    }
+                    m.base = p.probe_d[q * p.nprobe + m.pi];
+                }
+                ipm[tid] = m;
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int run = 0;
+                for (int i = 0; i < nt; ++i) {
+                    run += ipm[i].blk_end;
+                    ipm[i].blk_end = run;
+                }
+            }
+            __syncthreads();
+            if (DBG && p.masks) {
+                for (int i = tid; i < nt * nsub * 8; i += NT) {
+                    const IpProbe& m = ipm[i / (nsub * 8)];
+                    if (m.pi >= 0) p.masks[(q * p.nprobe + m.pi) * nsub * 8 + i % (nsub * 8)] = hitmask[i % (nsub * 8)];
+                }
+            }
+            const int total = ipm[nt - 1].blk_end;
+            int gb = warp, ci = 0;
+            while (true) {
+                const unsigned long long tau = *tau_p;
+                const uint32_t tau_hi = (uint32_t)(tau >> 32);
+                bool halt = false;
+#pragma unroll 1
+                for (; gb < total && !halt; gb += kWarps) {
+                    while (gb >= ipm[ci].blk_end) ++ci;   // gb only grows: the cursor follows it
+                    const IpProbe m = ipm[ci];
+                    const int first = ci > 0 ? ipm[ci - 1].blk_end : 0;
+                    halt = scan_block(std::integral_constant<int, 0>{}, gb - first, m.b0, m.len, m.p0, m.pi, m.base, tau, tau_hi);
+                }
+                if (!__syncthreads_or(gb < total || halt)) break;
+                topk_select<NT, CtaGroup, kCapN>(t, p.k);
+            }
+        }
+    }
+
+    if constexpr (!IP)
     for (int pi0 = split; pi0 < p.nprobe; pi0 += p.nsplit * NC) {
         // ---- the clusters of this phase; an invalid id leaves an empty list behind ----
         int cl[NC];
@@ -346,27 +525,19 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
             }
         }
         // (the barrier that ended the previous phase's scan makes the tables and `res` free)
+        if (!IP) {
 #pragma unroll
-        for (int k = 0; k < NC; ++k) {
-            const int c = cl[k] >= 0 ? cl[k] : 0;   // a table is built for every slot; an empty slot is never scanned
-            for (int j = tid; j < d; j += NT) res[k * dpad + j] = __fsub_rn(p.queries[q * d + j], p.cent[(int64_t)c * d + j]);
+            for (int k = 0; k < NC; ++k) {
+                const int c = cl[k] >= 0 ? cl[k] : 0;   // a table is built for every slot; an empty slot is never scanned
+                for (int j = tid; j < d; j += NT) res[k * dpad + j] = __fsub_rn(p.queries[q * d + j], p.cent[(int64_t)c * d + j]);
+            }
+            if (DBG)
+                for (int i = tid; i < NC * IVFPQ_MAX_NSUB * 8; i += NT) hitmask[i] = 0;
+            __syncthreads();
         }
-        if (DBG)
-            for (int i = tid; i < NC * IVFPQ_MAX_NSUB * 8; i += NT) hitmask[i] = 0;
-        __syncthreads();
 
-        // ---- selective tables, one per group and cluster ----
-        build_group<W0, DSUB, NT, DBG, SCORE_T, NC, GR::stride(0)>(lut, kSetFloats, p.cbt, res, dpad, r2, ksub, p.dense, p.score, P,
-                                                                  hitmask, IVFPQ_MAX_NSUB * 8);
-        if constexpr (W1 > 0)
-            build_group<W1, DSUB, NT, DBG, SCORE_T, NC, GR::stride(1)>(lut + GR::lut_off(1), kSetFloats,
-                                                                      p.cbt + (size_t)GR::s0(1) * 256 * DSUB, res + GR::s0(1) * DSUB, dpad,
-                                                                      r2 + GR::s0(1), ksub, p.dense, p.score, P,
-                                                                      hitmask + GR::s0(1) * 8, IVFPQ_MAX_NSUB * 8);
-        if constexpr (W2 > 0)
-            build_group<W2, DSUB, NT, DBG, SCORE_T, NC>(lut + GR::lut_off(2), kSetFloats, p.cbt + (size_t)GR::s0(2) * 256 * DSUB,
-                                                       res + GR::s0(2) * DSUB, dpad, r2 + GR::s0(2), ksub, p.dense, p.score, P,
-                                                       hitmask + GR::s0(2) * 8, IVFPQ_MAX_NSUB * 8);
+        // ---- selective tables, one per group and cluster (inner product: built once, above) ----
+        if (!IP) build_tables();
         __syncthreads();
         if (DBG && p.masks) {
 #pragma unroll
@@ -381,67 +552,19 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
         // ---- scan the lists of this phase as one sequence of blocks: the warp takes blocks warp,
         //      warp + kWarps, ...; block numbers at or beyond nblk[0] belong to the second list ----
         const int64_t nblk_all = NC == 2 ? nblk[0] + nblk[NC - 1] : nblk[0];
+        const float base = (IP && pi0 < p.nprobe) ? p.probe_d[q * p.nprobe + pi0] : 0.0f;   // inner product: -(q.c) of the cluster
         int64_t gb = warp;
         while (true) {
             const unsigned long long tau = *tau_p;
             const uint32_t tau_hi = (uint32_t)(tau >> 32);
             bool halt = false;
-            // one block of cluster slot K (a compile-time constant: the table bases are immediates)
-            auto scan_block = [&](auto slot_tag, int64_t blk) {
-                constexpr int K = decltype(slot_tag)::value;
-                bool stop = false;
-                const unsigned char* bp = reinterpret_cast<const unsigned char*>(p.codes_il) + (b0[K] + blk) * GR::kBlockBytes;
-                const float* lutk = lut + K * kSetFloats;
-                const uint32_t* hm = hitmask + K * IVFPQ_MAX_NSUB * 8;
-                uint32_t w0[W0 >= 4 ? W0 / 4 : 1];
-                uint32_t w1[W1 >= 4 ? W1 / 4 : 1];
-                uint32_t w2[W2 >= 4 ? W2 / 4 : 1];
-                (void)lutk; (void)w1; (void)w2;   // unused in the instances without those groups
-                load_group_codes<W0>(bp, lane, w0);
-                if constexpr (W1 > 0) load_group_codes<W1>(bp + GR::chunk_off(1), lane, w1);
-                if constexpr (W2 > 0) load_group_codes<W2>(bp + GR::chunk_off(2), lane, w2);
-                float acc = 0.0f;
-                unsigned long long hs = 0;
-                if constexpr (GR::kPaired) {
-                    float a0 = 0.0f, a1 = 0.0f;
-                    pair_gather_words<W0 / 4, (int)kWin + K * kSetBytes>(w0, pk, a0, a1);
-                    pair_gather_words<W1 / 4, (int)kWin + K * kSetBytes + 128>(w1, pk, a0, a1);
-                    acc = a0 + a1;
-                    if (DBG) {
-                        hits_group<W0>(w0, lane, 0, hm, hs);
-                        hits_group<W1>(w1, lane, GR::s0(1), hm, hs);
-                    }
-                } else {
-                    gather_group<W0, DBG>(lutk, w0, lane, 0, hm, acc, hs);
-                    if constexpr (W1 > 0) gather_group<W1, DBG>(lutk + GR::lut_off(1), w1, lane, GR::s0(1), hm, acc, hs);
-                }
-                if constexpr (W2 > 0) gather_group<W2, DBG>(lutk + GR::lut_off(2), w2, lane, GR::s0(2), hm, acc, hs);
-                const int64_t pos = blk * kPointsPerBlock + lane;
-                if (pos < len[K]) {
-                    if (DBG) {
-                        const int64_t vi = vprefix[pi0 + K * p.nsplit] + pos;
-                        if (vi < p.visit_stride) {
-                            if (p.visit_hits) p.visit_hits[q * p.visit_stride + vi] = hs;
-                            if (p.visit_dist) p.visit_dist[q * p.visit_stride + vi] = acc;
-                            if (p.visit_ids) p.visit_ids[q * p.visit_stride + vi] = p.ids[p0[K] + pos];
-                        }
-                    }
-                    if (__float_as_uint(acc) <= tau_hi) {
-                        const unsigned long long key = make_key(acc, (uint32_t)p.ids[p0[K] + pos]);
-                        if (key < tau) {
-                            const int slot = atomicAdd(cnt_p, 1);
-                            if (slot < kCapN) kbuf[slot] = key;
-                            else atomicOr(p.status, kFlagOverflow);
-                            stop = slot >= kSoft;
-                        }
-                    }
-                }
-                return __any_sync(0xFFFFFFFFu, stop);
-            };
 #pragma unroll 1
             for (; gb < nblk_all && !halt; gb += kWarps) {
-                if (NC == 1 || gb < nblk[0]) halt = scan_block(std::integral_constant<int, 0>{}, gb);
-                else halt = scan_block(std::integral_constant<int, NC - 1>{}, gb - nblk[0]);
+                if (NC == 1 || gb < nblk[0])
+                    halt = scan_block(std::integral_constant<int, 0>{}, gb, b0[0], len[0], p0[0], pi0, base, tau, tau_hi);
+                else
+                    halt = scan_block(std::integral_constant<int, NC - 1>{}, gb - nblk[0], b0[NC - 1], len[NC - 1], p0[NC - 1],
+                                      pi0 + (NC - 1) * p.nsplit, 0.0f, tau, tau_hi);
             }
             // The barrier that ends the phase (tables free for the next one).  A set flag means that a
             // warp met the soft limit (it may have finished its blocks all the same): the buffer is
@@ -464,21 +587,21 @@ __global__ void __launch_bounds__(NT, NT == 512 ? 2 : 1) scan_rot_kernel(const S
     const int n = min(*cnt_p, p.k);
     if (p.nsplit == 1) {
         for (int i = tid; i < p.k; i += NT) {
-            const unsigned long long key = i < n ? kbuf[i] : kKeyPad;
-            p.out_dist[q * p.k + i] = __uint_as_float((uint32_t)(key >> 32));
+            const unsigned long long key = i < n ? kbuf[i] : t.pad;
+            p.out_dist[q * p.k + i] = IP ? -from_ordered_bits((uint32_t)(key >> 32)) : __uint_as_float((uint32_t)(key >> 32));
             p.out_ids[q * p.k + i] = (int32_t)(uint32_t)(key & 0xFFFFFFFFull);
         }
     } else {
         unsigned long long* dst = p.partial + (q * p.nsplit + split) * p.k;
-        for (int i = tid; i < p.k; i += NT) dst[i] = i < n ? kbuf[i] : kKeyPad;
+        for (int i = tid; i < p.k; i += NT) dst[i] = i < n ? kbuf[i] : t.pad;
     }
 }
 
-template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T, int NC>
+template <int W0, int W1, int W2, int DSUB, int NT, bool DBG, int SCORE_T, int NC, bool IP = false>
 cudaError_t launch_rot_inst(const ScanParams& sp, int64_t grid, int nprobe, cudaStream_t st) {
     const size_t smem = rot_smem_bytes(Groups<W0, W1, W2>::kPaired, (((Groups<W0, W1, W2>::kLutFloats * 4 + 255) / 256) * 256) / 4, sp.d,
-                                       nprobe, DBG, NC);
-    auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, DBG, SCORE_T, NC>;
+                                       nprobe, DBG, NC, IP);
+    auto kern = scan_rot_kernel<W0, W1, W2, DSUB, NT, DBG, SCORE_T, NC, IP>;
     const cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<(unsigned)grid, NT, smem, st>>>(sp);
@@ -494,6 +617,13 @@ cudaError_t launch_rot(const ScanParams& sp, int64_t grid, bool debug, int nprob
     if (sp.score == IVFPQ_SCORE_REWARD_PENALTY)
         return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_REWARD_PENALTY, NC>(sp, grid, nprobe, st);
     return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_DISTANCE, NC>(sp, grid, nprobe, st);
+}
+
+// Inner product: distances only (one production instance, one with stage dumps).
+template <int W0, int W1, int W2, int DSUB, int NT>
+cudaError_t launch_rot_ip(const ScanParams& sp, int64_t grid, bool debug, int nprobe, cudaStream_t st) {
+    if (debug) return launch_rot_inst<W0, W1, W2, DSUB, NT, true, IVFPQ_SCORE_DISTANCE, 1, true>(sp, grid, nprobe, st);
+    return launch_rot_inst<W0, W1, W2, DSUB, NT, false, IVFPQ_SCORE_DISTANCE, 1, true>(sp, grid, nprobe, st);
 }
 
 }  // namespace
@@ -527,6 +657,14 @@ cudaError_t launch_scan_rot(const ivfpq_index* ix, const ScanParams& sp, int64_t
     // probed clusters per pass over the codebook) halves the codebook traffic but measured slower
     // (48 x 2: 4.0 -> 5.2 ms, 50 x 4: 12.1 -> 13.8 ms): one CTA's 32 warps meet at every barrier,
     // where two independent CTAs of 16 warps overlap.
+    if (ix->metric == IVFPQ_METRIC_IP) {
+        if (ix->nsub == 16 && ix->dsub == 8) return launch_rot_ip<16, 0, 0, 8, 512>(sp, grid, debug, nprobe, st);
+        if (ix->nsub == 48 && ix->dsub == 2) return launch_rot_ip<32, 16, 0, 2, 512>(sp, grid, debug, nprobe, st);
+        if (ix->nsub == 50 && ix->dsub == 4) return launch_rot_ip<32, 16, 2, 4, 512>(sp, grid, debug, nprobe, st);
+        if (ix->nsub == 8 && ix->dsub == 4) return launch_rot_ip<8, 0, 0, 4, 256>(sp, grid, debug, nprobe, st);
+        if (ix->nsub == 12 && ix->dsub == 2) return launch_rot_ip<8, 4, 0, 2, 256>(sp, grid, debug, nprobe, st);
+        return cudaErrorNotSupported;
+    }
     const bool pair = ix->rot_pair != 0;
     if (ix->nsub == 48 && ix->dsub == 2)
         return pair ? launch_rot<32, 16, 0, 2, 1024, 2>(sp, grid, debug, nprobe, st) : launch_rot<32, 16, 0, 2, 512, 1>(sp, grid, debug, nprobe, st);
