@@ -113,6 +113,31 @@ def test_inner_product_search_matches_oracle(shaped, name):
 
 
 @pytest.mark.parametrize("name", [s[0] for s in SHAPES])
+def test_inner_product_more_probes_than_one_staged_tile(shaped, name):
+    """80 and 96 probed clusters (all of them): the kernels of the conflict-free layouts stage the list
+    metadata of 64 clusters at a time and scan a tile's lists as one block sequence; alone and split
+    over several CTAs per query, with stage dumps for a few queries."""
+    wl, idx, h = shaped[name]
+    q = dev(wl.queries)
+    floor = magnitude(idx, wl.queries)
+    for nsplit in (0, 5):
+        lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_NSPLIT, nsplit)
+        for nprobe in sorted({min(80, idx.nlist), idx.nlist}):
+            d, i = lib.ivfpq_search_sparse(h, q, nprobe, dev(wl.radius), 100, scale=1.5)
+            assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
+            check(d, i, oracle.search(idx, wl.queries, nprobe, 100, radius=wl.radius, scale=1.5), floor)
+    lib.ivfpq_index_set_option(h, lib.IVFPQ_OPT_NSPLIT, 0)
+    nq, nprobe = 6, min(70, idx.nlist)
+    stride = int(np.diff(idx.list_offsets).max()) * nprobe
+    g = lib.ivfpq_debug_search(h, dev(wl.queries[:nq]), nprobe, 50, radius=dev(wl.radius), scale=1.5, visit_stride=stride)
+    assert lib.ivfpq_sync_status(h) == lib.IVFPQ_OK
+    g = {k2: host(v) for k2, v in g.items()}
+    o = oracle.search(idx, wl.queries[:nq], nprobe, 50, radius=wl.radius, scale=1.5, dumps=True, visit_stride=stride)
+    assert np.array_equal(g["masks"].view(np.uint32), o["masks"])
+    assert_visits_parity(g, o, idx.nsub, floor=magnitude(idx, wl.queries[:nq]))
+
+
+@pytest.mark.parametrize("name", [s[0] for s in SHAPES])
 def test_inner_product_stage_dumps(shaped, name):
     wl, idx, h = shaped[name]
     nq, nprobe, stride = 24, 5, 6000
