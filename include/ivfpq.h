@@ -91,7 +91,9 @@ typedef struct {
 } ivfpq_index_desc_t;
 
 /* Bytes of caller-owned device memory that ivfpq_index_load needs for derived tables (codes
- * re-laid-out in 32-point interleaved blocks, list tables, the smallest id of every block; for the 16 x 8 shape under L2 also the
+ * re-laid-out in 32-point interleaved blocks, list tables, the smallest id of every block, for the
+ * tensor-core filtering the centroids' squared norms and, under L2, a copy of the centroids with their
+ * mean subtracted; for the 16 x 8 shape under L2 also the
  * inverted index from codebook entries to points of Algorithm 1, 2 bytes per code byte plus
  * 16 KB per 8192 points of a list).  0 on invalid descriptions. */
 size_t ivfpq_index_derived_bytes(const ivfpq_index_desc_t* desc);

@@ -59,7 +59,7 @@ int plan_derived(const ivfpq_index_desc_t* d, DerivedLayout* out) {
     if (out->rot) off = align_up(off + (size_t)d->nsub * 256 * d->dsub * 4, 256);
     out->cnorm_off = off;
     out->mma = coarse_mma_supported(d->d, d->nlist) ? 1 : 0;
-    if (out->mma) off = align_up(off + coarse_mma_derived_bytes(d->nlist), 256);
+    if (out->mma) off = align_up(off + coarse_mma_derived_bytes(d->nlist, d->d, d->metric == IVFPQ_METRIC_L2), 256);
     out->blk_min_off = off;
     off = align_up(off + (size_t)nblocks * 4, 256);
     // entry -> points map of the sparsity-aware scan: the 16 x 8 shape under L2 (element indices are 32-bit)
@@ -175,7 +175,7 @@ WorkspaceLayout plan_workspace(const ivfpq_index* ix, int64_t nq, int32_t nprobe
     wl.probe_d_off = off;
     off = align_up(off + (size_t)nq * nprobe * 4, 256);
     wl.coarse_off = off;
-    off = align_up(off + (size_t)qchunk * ix->nlist * 4, 256);
+    off = align_up(off + coarse_region_bytes(ix, qchunk), 256);
     wl.partial_off = off;
     // sized for the largest split the option may select later, so that the option can change
     // without a new workspace query
@@ -249,6 +249,13 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
     ix->block_bytes = dl.block_bytes;
     ix->cbt = reinterpret_cast<const float*>(base + dl.cbt_off);
     ix->cnorm = dl.mma ? reinterpret_cast<const float*>(base + dl.cnorm_off) : nullptr;
+    {
+        // behind the norms and their maximum: the centroids' mean and the centred centroids (L2 only)
+        const bool centered = dl.mma && desc->metric == IVFPQ_METRIC_L2;
+        char* at = base + dl.cnorm_off + align_up((size_t)desc->nlist * 4, 256) + 256;
+        ix->mu = centered ? reinterpret_cast<const float*>(at) : nullptr;
+        ix->cent_c = centered ? reinterpret_cast<const float*>(at + align_up((size_t)desc->d * 4, 256)) : nullptr;
+    }
     ix->max_list_len = dl.max_len;
     ix->blk_min = reinterpret_cast<const uint32_t*>(base + dl.blk_min_off);
     ix->chunk_first = dl.map ? reinterpret_cast<const int32_t*>(base + dl.chunk_first_off) : nullptr;
@@ -301,8 +308,10 @@ int ivfpq_index_load(const ivfpq_index_desc_t* desc, void* derived_dev, size_t d
                             reinterpret_cast<float*>(base + dl.cbt_off), st);
     if (e == cudaSuccess) e = launch_block_min_id(ix, reinterpret_cast<uint32_t*>(base + dl.blk_min_off), st);
     if (e == cudaSuccess) e = launch_entry_map(ix, desc->codes, st);
+    if (e == cudaSuccess && ix->cent_c)
+        e = launch_center(ix->cent, ix->nlist, ix->d, const_cast<float*>(ix->mu), const_cast<float*>(ix->cent_c), st);
     if (e == cudaSuccess && ix->cnorm)
-        e = launch_cnorm(ix->cent, ix->nlist, ix->d, reinterpret_cast<float*>(base + dl.cnorm_off), st);
+        e = launch_cnorm(ix->cent_c ? ix->cent_c : ix->cent, ix->nlist, ix->d, reinterpret_cast<float*>(base + dl.cnorm_off), st);
     if (e != cudaSuccess) {
         delete ix;
         return IVFPQ_ERR_CUDA;

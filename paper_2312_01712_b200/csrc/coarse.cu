@@ -140,19 +140,32 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
     const bool mma_shape = ix->cnorm != nullptr && (reinterpret_cast<uintptr_t>(queries) & 15) == 0 &&
                            (reinterpret_cast<uintptr_t>(ix->cent) & 15) == 0;
     const int64_t qchunk_row = qchunk;   // queries whose full rows fit the scratch region (the plain kernels need those)
+    const size_t region = coarse_region_bytes(ix, qchunk);   // bytes of scratch the caller provides
     bool mma = mma_shape, fused = false;
-    if (mma && coarse_mma_fused(ix->nlist, nprobe) && !ix->test_fault) {
-        // the fused path needs another amount of scratch per query than a full row: its own chunking of the same region
-        const int64_t fit = (int64_t)(((size_t)qchunk * ix->nlist * 4) / coarse_mma_fused_bytes_per_query(ix->nlist));
-        if (fit >= 1) {
-            qchunk = fit < nq ? fit : nq;   // more queries per chunk than full rows would allow, or fewer
-            fused = true;
+    // L2: the proposal works on centred operands; the centred queries of a chunk take d floats each at
+    // the front of the same region (no centring when not even one query fits that way)
+    const size_t qc_bytes = (mma && ix->cent_c) ? (size_t)ix->d * 4 : 0;
+    bool centred = qc_bytes != 0;
+    if (mma) {
+        if (coarse_mma_fused(ix->nlist, nprobe) && !ix->test_fault) {
+            // the fused path needs another amount of scratch per query than a full row: its own chunking of the same region
+            const int64_t fit = (int64_t)((region > 256 ? region - 256 : 0) / (coarse_mma_fused_bytes_per_query(ix->nlist) + qc_bytes));   // 256: alignment of the second part
+            if (fit >= 1) {
+                qchunk = fit < nq ? fit : nq;   // more queries per chunk than full rows would allow, or fewer
+                fused = true;
+            }
+        }
+        if (!fused && centred) {
+            // (full rows and centred queries of `qchunk` queries fit by the region's definition)
         }
     }
     for (int64_t q0 = 0; q0 < nq; q0 += qchunk) {
         int nqc = (int)((nq - q0 < qchunk) ? (nq - q0) : qchunk);
         if (mma) {
-            const cudaError_t e = launch_coarse_mma(ix, queries, q0, nqc, nprobe, fused, coarse_tile, probe_ids, probe_d, status, st, launches);
+            // [centred queries of the chunk][tile rows, or the fused path's scratch]: both 256-byte aligned
+            float* q_centred = centred ? coarse_tile : nullptr;
+            float* tile = centred ? reinterpret_cast<float*>(reinterpret_cast<char*>(coarse_tile) + align_up((size_t)qchunk * qc_bytes, 256)) : coarse_tile;
+            const cudaError_t e = launch_coarse_mma(ix, queries, q0, nqc, nprobe, fused, q_centred, tile, probe_ids, probe_d, status, st, launches);
             if (e == cudaSuccess) continue;
             if (e != cudaErrorNotSupported) return e;
             mma = false;   // the tensor maps could not be built: the plain kernels, in chunks of full rows
@@ -222,7 +235,8 @@ extern "C" int ivfpq_probe_static(const ivfpq_index_t* index, const float* queri
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     // the status word must start at zero; the tile is fully rewritten before it is read
     if (cudaMemsetAsync(scratch, 0, 256, st) != cudaSuccess) return IVFPQ_ERR_CUDA;
-    int64_t qchunk = ((int64_t)IVFPQ_STATIC_SCRATCH_BYTES - 256) / ((int64_t)index->nlist * 4);
+    // status word, then the filtering stage's region for chunks of qchunk queries (coarse_region_bytes)
+    int64_t qchunk = ((int64_t)IVFPQ_STATIC_SCRATCH_BYTES - 512) / ((int64_t)index->nlist * 4 + (int64_t)index->d * 4);
     if (qchunk > nq) qchunk = nq;
     int64_t launches = 0;
     if (ivfpq::launch_coarse(index, queries, nq, nprobe, reinterpret_cast<float*>(scratch + 256), qchunk,

@@ -3,7 +3,9 @@
 //
 // The tensor cores only *propose*: the nprobe closest clusters are decided by the defining fp32
 // arithmetic (sum over dimensions of fma(t, t, acc), t = q_j - c_j, j ascending), because the probe
-// lists must not depend on how a GEMM rounds.
+// lists must not depend on how a GEMM rounds.  Under L2 they work on centred operands (queries and
+// centroids minus the centroids' mean: the distance is the same, the norms - and with them the error
+// bound of the TF32 products - are smaller); the exact decision keeps the original vectors.
 //
 //   1. coarse_mma_kernel: approx[q][c] = |c|^2 - 2 q.c for a tile of queries against all centroids.
 //      TMA (cp.async.bulk.tensor, 128-byte swizzle) stages fp32 tiles of queries and centroids in
@@ -382,6 +384,43 @@ __global__ void __launch_bounds__(256) cnorm_kernel(const float* __restrict__ ce
     atomicMax(cmax_bits, __float_as_uint(s));
 }
 
+// Centring of the proposal's operands (L2 only).  A squared distance does not change when the same
+// vector is subtracted from the query and from the centroid, while the error of the TF32 products
+// scales with the norms of the factors: the tensor cores therefore work on q - mu and c - mu, mu the
+// mean of the centroids (any fixed vector would do; its rounding does not matter).  The exact decision
+// keeps the original vectors.
+__global__ void __launch_bounds__(256) centroid_mean_kernel(const float* __restrict__ cent, int nlist, int d,
+                                                            float* __restrict__ mu) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= d) return;
+    float s = 0.0f;
+    for (int c = 0; c < nlist; ++c) s += cent[(size_t)c * d + j];
+    mu[j] = s / (float)nlist;
+}
+
+// out[r][j] = in[r][j] - mu[j]
+__global__ void __launch_bounds__(256) subtract_mean_kernel(const float* __restrict__ in, const float* __restrict__ mu,
+                                                            int64_t n, int d, float* __restrict__ out) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) out[i] = __fsub_rn(in[i], mu[i % d]);
+}
+
+// |approx - exact| <= eps for the tile value of one (query, centroid) pair.  qn, cmax: squared norm of
+// the query and largest squared norm of a centroid AS THE TENSOR CORES SAW THEM (centred for L2).
+// First term: TF32 keeps 10 mantissa bits of each factor (relative 2^-10 each, 2^-9 per product),
+// summed over the dimensions by Cauchy-Schwarz and doubled by the factor -2 (inner product: the cost
+// is half the tile value).  Second term, fp32 rounding.  L2, centred operands q' = fl(q - mu),
+// c' = fl(c - mu): the tensor-core accumulation (d), the two squared norms (d + 1 each), the final
+// additions, the exact chain on the other side ((d + 2) on |q - c|^2 <= 2 (|q'|^2 + |c'|^2)) and the
+// rounding of the centring itself (2^-22 (|q'|^2 + |c'|^2)), each at most 2^-24 of that magnitude per
+// operation: (4 d + 17) 2^-24 (|q'|^2 + |c'|^2), taken as 4 d + 32.  Inner product (not centred): the
+// accumulation on both sides, on |q||c|.
+__device__ __forceinline__ float proposal_eps(bool ip, float qn, float cmax, int d) {
+    const float qc = sqrtf(qn) * sqrtf(cmax);
+    return ip ? 0.625f * 0.00390625f * qc + (float)(2 * d + 8) * 5.9604645e-8f * qc
+              : 1.25f * 0.00390625f * qc + (float)(4 * d + 32) * 5.9604645e-8f * (qn + cmax);
+}
+
 // One CTA per query: cut from the approximate distances, exact re-evaluation of everything under
 // the cut, the nprobe smallest (distance, cluster id) ascending.
 template <bool IP>
@@ -390,7 +429,8 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
                                                           int nlist, int d, int nprobe, int64_t q0,
                                                           int32_t* __restrict__ probe_ids, float* __restrict__ probe_d,
                                                           int* __restrict__ status, const uint2* __restrict__ clist,
-                                                          const int* __restrict__ ccount, int ccap) {
+                                                          const int* __restrict__ ccount, int ccap, const float* __restrict__ mu) {
+    // mu != null: the tile values come from centred operands; qn is then |q - mu|^2
     // clist != null: the proposals are the (value, cluster) pairs the filtering epilogue kept for this
     // query instead of a full row; a list that did not fit means: evaluate every cluster exactly.
     extern __shared__ __align__(1024) unsigned char dyn[];
@@ -418,7 +458,8 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
     for (int j = tid; j < d; j += 256) {
         const float x = queries[q * d + j];
         qs[j] = x;
-        part = fmaf(x, x, part);
+        const float xc = mu ? __fsub_rn(x, mu[j]) : x;
+        part = fmaf(xc, xc, part);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
@@ -430,15 +471,7 @@ __global__ void __launch_bounds__(256) probe_rerank_kernel(const float* __restri
 #pragma unroll
     for (int i = 0; i < 8; ++i) qn += red[i];
     const float cmax = __uint_as_float(*cmax_bits);
-    // |approx - exact| <= eps: TF32 keeps 10 mantissa bits of each factor (relative 2^-10 each, 2^-9
-    // per product), summed over the dimensions by Cauchy-Schwarz and doubled by the factor -2; the
-    // second term covers the fp32 rounding of both sides, which grows with the number of summed
-    // terms: d accumulations in the tensor-core sum and in the squared norms, d in the exact chain
-    // (each at most 2^-24 of the running magnitude, itself at most |q|^2 + max|c|^2 up to a factor 2).
-    // Inner product: the approximate cost is -q.c = half the tile value; half the TF32 term, and the
-    // rounding term on |q||c| instead of the norms.
-    const float eps = IP ? 0.625f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * sqrtf(qn) * sqrtf(cmax)
-                         : 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
+    const float eps = proposal_eps(IP, qn, cmax, d);
     // what the two sides are ranked by: squared distance (tile value + |q|^2, clamped at 0), or the cost -q.c
     auto approx_of = [&](float v) { return IP ? 0.5f * v : fmaxf(v + qn, 0.0f); };
     auto key_of = [&](float x, int id) {
@@ -565,7 +598,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kerne
     const float* __restrict__ approx, const float* __restrict__ queries, const float* __restrict__ cent,
     const unsigned* __restrict__ cmax_bits, int nlist, int d, int nprobe, int64_t q0, int nqc,
     int32_t* __restrict__ probe_ids, float* __restrict__ probe_d, const uint2* __restrict__ clist,
-    const int* __restrict__ ccount, int ccap) {
+    const int* __restrict__ ccount, int ccap, const float* __restrict__ mu) {
     // clist != null: the proposals are the (value, cluster) pairs the filtering epilogue kept for the
     // query (at most ccap <= kWarpRowMax); a list that did not fit, or is shorter than nprobe, means:
     // every cluster is evaluated exactly
@@ -595,15 +628,14 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kerne
     for (int j = lane; j < d; j += 32) {
         const float x = queries[q * d + j];
         qs[j] = x;
-        part = fmaf(x, x, part);
+        const float xc = mu ? __fsub_rn(x, mu[j]) : x;   // centred operands: |q - mu|^2
+        part = fmaf(xc, xc, part);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, o);
     const float qn = part;
     const float cmax = __uint_as_float(*cmax_bits);
-    // the error bound of probe_rerank_kernel (any order of the |q|^2 sum is covered by its second term)
-    const float eps = IP ? 0.625f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * sqrtf(qn) * sqrtf(cmax)
-                         : 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) + (float)(2 * d + 8) * 5.9604645e-8f * (qn + cmax);
+    const float eps = proposal_eps(IP, qn, cmax, d);   // (any order of the |q|^2 sum is covered by its second term)
     __syncwarp();
 
     // what a cluster is proposed by, as bits whose unsigned order is the order of the values:
@@ -787,7 +819,8 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 8) probe_rerank_warp_kerne
 constexpr int kBoundPerThread = 16;
 __global__ void __launch_bounds__(256) probe_bound_kernel(const float* __restrict__ sample, int m, const float* __restrict__ queries,
                                                          const unsigned* __restrict__ cmax_bits, int d, int nprobe, int64_t q0,
-                                                         float* __restrict__ cutp, int* __restrict__ ccount, int ip) {
+                                                         float* __restrict__ cutp, int* __restrict__ ccount, int ip,
+                                                         const float* __restrict__ mu) {
     __shared__ int hist[256];
     __shared__ int wsum[8];
     __shared__ unsigned mm[2];
@@ -810,7 +843,8 @@ __global__ void __launch_bounds__(256) probe_bound_kernel(const float* __restric
     float qn = 0.0f;
     for (int j = tid; j < d; j += 256) {
         const float x = queries[(q0 + ql) * d + j];
-        qn = fmaf(x, x, qn);
+        const float xc = mu ? __fsub_rn(x, mu[j]) : x;
+        qn = fmaf(xc, xc, qn);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) qn += __shfl_xor_sync(0xFFFFFFFFu, qn, o);
@@ -873,8 +907,7 @@ __global__ void __launch_bounds__(256) probe_bound_kernel(const float* __restric
         const float kth = from_ordered_bits(top);   // at or above the nprobe-th smallest sampled value
         const float cmax = __uint_as_float(*cmax_bits);
         // error bound of the tile value: |c|^2 - 2 q.c against the squared distance, or -2 q.c against twice the cost
-        const float eps = 1.25f * 0.00390625f * sqrtf(qn) * sqrtf(cmax) +
-                          (float)(2 * d + 8) * 5.9604645e-8f * (ip ? 2.0f * sqrtf(qn) * sqrtf(cmax) : qn + cmax);
+        const float eps = ip ? 2.0f * proposal_eps(true, qn, cmax, d) : proposal_eps(false, qn, cmax, d);
         cutp[ql] = kth + 2.0f * eps + 1e-6f * fabsf(kth);   // the last term: the two sides add |q|^2 in different places
         ccount[ql] = 0;
     }
@@ -915,7 +948,20 @@ bool coarse_mma_supported(int d, int nlist) {
     return d % 4 == 0 && d >= 4 && (d + kKBlock - 1) / kKBlock <= kMaxKBlocks && nlist >= 1 && encode_tiled_fn() != nullptr;
 }
 
-size_t coarse_mma_derived_bytes(int nlist) { return align_up((size_t)nlist * 4, 256) + 256; }
+// norms | their maximum | (L2) mean of the centroids | centred centroids
+size_t coarse_mma_derived_bytes(int nlist, int d, bool centered) {
+    size_t b = align_up((size_t)nlist * 4, 256) + 256;
+    if (centered) b += align_up((size_t)d * 4, 256) + align_up((size_t)nlist * d * 4, 256);
+    return b;
+}
+
+// mu = mean of the centroids, cent_c = cent - mu (derived buffer of an L2 index).
+cudaError_t launch_center(const float* cent, int nlist, int d, float* mu, float* cent_c, cudaStream_t st) {
+    centroid_mean_kernel<<<(d + 255) / 256, 256, 0, st>>>(cent, nlist, d, mu);
+    const int64_t n = (int64_t)nlist * d;
+    subtract_mean_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(cent, mu, n, d, cent_c);
+    return cudaGetLastError();
+}
 
 // Fills cnorm[nlist] and the max word behind it (derived buffer of the index).
 cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st) {
@@ -949,11 +995,18 @@ size_t coarse_mma_fused_bytes_per_query(int nlist) { return (size_t)sample_clust
 // tensor maps cannot be built (the caller then uses the plain kernels).  `tile` is scratch of at
 // least nqc * nlist floats (full-tile path) or, with `fused`, nqc * coarse_mma_fused_bytes_per_query() bytes.
 cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe, bool fused,
-                              float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
+                              float* q_centered, float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
                               int64_t* launches) {
+    // L2 with room for the centred queries (nqc x d floats): the proposal works on centred operands
+    const float* mu = (ix->cent_c && q_centered) ? ix->mu : nullptr;
     alignas(64) CUtensorMap map_q, map_c;
-    if (!make_map(&map_q, queries + q0 * ix->d, nqc, ix->d)) return cudaErrorNotSupported;
-    if (!make_map(&map_c, ix->cent, ix->nlist, ix->d)) return cudaErrorNotSupported;
+    if (!make_map(&map_q, mu ? q_centered : queries + q0 * ix->d, nqc, ix->d)) return cudaErrorNotSupported;
+    if (!make_map(&map_c, mu ? ix->cent_c : ix->cent, ix->nlist, ix->d)) return cudaErrorNotSupported;
+    if (mu) {
+        const int64_t n = (int64_t)nqc * ix->d;
+        subtract_mean_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(queries + q0 * ix->d, mu, n, ix->d, q_centered);
+        *launches += 1;
+    }
     const int kblocks = (ix->d + kKBlock - 1) / kKBlock;
     const int qtiles = (nqc + kTileM - 1) / kTileM;
     const int ntile = (ix->nlist + kTileN - 1) / kTileN;
@@ -986,7 +1039,7 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
         const int stile = nsample / kTileN;
         coarse_mma_kernel<<<dim3(qtiles, csplit_for(stile)), kMmaThreads, smem, st>>>(
             map_q, map_c, cnorm, nqc, ix->nlist, kblocks, sample, status, 0, stile, nsample, nullptr, nullptr, nullptr, 0, nstages, ip);
-        probe_bound_kernel<<<nqc, 256, 0, st>>>(sample, nsample, queries, cmax, ix->d, nprobe, q0, cutp, ccount, ip);
+        probe_bound_kernel<<<nqc, 256, 0, st>>>(sample, nsample, queries, cmax, ix->d, nprobe, q0, cutp, ccount, ip, mu);
         coarse_mma_kernel<<<dim3(qtiles, csplit_for(ntile)), kMmaThreads, smem, st>>>(
             map_q, map_c, cnorm, nqc, ix->nlist, kblocks, nullptr, status, 0, ntile, 0, cutp, ccount, clist, kListCap, nstages, ip);
         if (nprobe <= kWarpCand / 2 && nprobe < ix->nlist && kListCap <= kWarpRowMax) {
@@ -994,10 +1047,10 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
             const size_t smem3 = (size_t)kWarpsPerCta * warp_rerank_smem_per_warp(ix->d);
             auto by_warp_kernel = ip ? probe_rerank_warp_kernel<true> : probe_rerank_warp_kernel<false>;
             by_warp_kernel<<<(nqc + kWarpsPerCta - 1) / kWarpsPerCta, kWarpKernelThreads, smem3, st>>>(
-                nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d, clist, ccount, kListCap);
+                nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d, clist, ccount, kListCap, mu);
         } else {
             rerank<<<nqc, 256, smem2, st>>>(nullptr, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
-                                                          probe_d, status, clist, ccount, kListCap);
+                                                          probe_d, status, clist, ccount, kListCap, mu);
         }
         *launches += 4;
         return cudaGetLastError();
@@ -1012,10 +1065,10 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
         const size_t smem3 = (size_t)kWarpsPerCta * warp_rerank_smem_per_warp(ix->d);
         auto by_warp_kernel = ip ? probe_rerank_warp_kernel<true> : probe_rerank_warp_kernel<false>;
         by_warp_kernel<<<(nqc + kWarpsPerCta - 1) / kWarpsPerCta, kWarpKernelThreads, smem3, st>>>(
-            tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d, nullptr, nullptr, 0);
+            tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, nqc, probe_ids, probe_d, nullptr, nullptr, 0, mu);
     } else {
         rerank<<<nqc, 256, smem2, st>>>(tile, queries, ix->cent, cmax, ix->nlist, ix->d, nprobe, q0, probe_ids,
-                                                      probe_d, status, nullptr, nullptr, 0);
+                                                      probe_d, status, nullptr, nullptr, 0, mu);
     }
     *launches += 2;
     return cudaGetLastError();

@@ -48,6 +48,9 @@ struct ivfpq_index {
     int32_t block_bytes;      // bytes of one 32-point code block in the rotated layout
     const float* cbt;         // [group][entry 0..255][column][dsub]
     const float* cnorm;       // [nlist] squared centroid norms + their maximum (tensor-core filtering), or null
+    const float* mu;          // [d] mean of the centroids, and
+    const float* cent_c;      // [nlist][d] centroids minus that mean: the tensor-core proposal of an L2 index works on these
+                              // (cnorm then holds their norms); null for the inner product
     // entry -> points map (entry_map.cu; 16 x 8 shape under L2 only, null otherwise)
     const int32_t* chunk_first;  // [nlist+1] chunks before each list
     const uint32_t* map_off;     // [nchunks][nsub][256]: first position | point count << 16 of every entry
@@ -76,6 +79,11 @@ struct ivfpq_index {
 namespace ivfpq {
 
 // Shape served by the persistent kernels (scan16x8.cu).
+// Scratch of the filtering stage for chunks of `qchunk` queries: a [qchunk][nlist] tile of proposed
+// values (or the fused path's smaller per-query scratch) and the centred queries of the chunk.
+inline size_t coarse_region_bytes(const ivfpq_index* ix, int64_t qchunk) {
+    return (size_t)qchunk * ((size_t)ix->nlist * 4 + (size_t)ix->d * 4) + 256;
+}
 inline bool pers_shape(const ivfpq_index* ix) { return ix->rot && ix->nsub == 16 && ix->dsub == 8; }
 
 struct SearchArgs {
@@ -127,13 +135,14 @@ int rot_block_bytes(const int w[3]);
 bool rot_supported(int nsub, int dsub);
 // Tensor-core filtering (coarse_mma.cu).
 bool coarse_mma_supported(int d, int nlist);
-size_t coarse_mma_derived_bytes(int nlist);
+size_t coarse_mma_derived_bytes(int nlist, int d, bool centered);
 bool coarse_mma_fused(int nlist, int nprobe);
 size_t coarse_mma_fused_bytes_per_query(int nlist);
 cudaError_t launch_entry_map(const ivfpq_index* ix, const uint8_t* codes, cudaStream_t st);
 cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st);
+cudaError_t launch_center(const float* cent, int nlist, int d, float* mu, float* cent_c, cudaStream_t st);
 cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64_t q0, int nqc, int32_t nprobe, bool fused,
-                              float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
+                              float* q_centered, float* tile, int32_t* probe_ids, float* probe_d, int* status, cudaStream_t st,
                               int64_t* launches);
 cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t nq, int32_t nprobe,
                           float* coarse_tile, int64_t qchunk, int32_t* probe_ids, float* probe_d,
