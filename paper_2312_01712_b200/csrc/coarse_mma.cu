@@ -1010,10 +1010,22 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
     const int kblocks = (ix->d + kKBlock - 1) / kKBlock;
     const int qtiles = (nqc + kTileM - 1) / kTileM;
     const int ntile = (ix->nlist + kTileN - 1) / kTileN;
+    // Into how many CTAs the centroid tiles of one query tile are split: one CTA per SM (shared memory),
+    // so the grid runs in waves of sm_count CTAs; the split with the fewest (waves x tiles per CTA,
+    // one more tile's worth per CTA for its start-up) wins.  (Rounding the split up to "about two
+    // waves" gave 308 CTAs on 148 SMs for 22 query tiles: a third wave of 12 CTAs.)
     auto csplit_for = [&](int tiles) {
-        int cs = (2 * ix->sm_count + qtiles - 1) / qtiles;   // about two waves of CTAs
-        if (cs > tiles) cs = tiles;
-        return cs < 1 ? 1 : cs;
+        int best = 1;
+        long best_cost = -1;
+        for (int cs = 1; cs <= tiles && cs <= 4 * ix->sm_count; ++cs) {
+            const long waves = ((long)qtiles * cs + ix->sm_count - 1) / ix->sm_count;
+            const long cost = waves * ((tiles + cs - 1) / cs + 1);
+            if (best_cost < 0 || cost < best_cost) {
+                best_cost = cost;
+                best = cs;
+            }
+        }
+        return best;
     };
     int nstages = 12 - kblocks;   // 16 KB tiles: queries + stages within about 200 KB
     if (nstages > kStages) nstages = kStages;
