@@ -149,7 +149,7 @@ cudaError_t launch_coarse(const ivfpq_index* ix, const float* queries, int64_t n
     if (mma) {
         if (coarse_mma_fused(ix->nlist, nprobe) && !ix->test_fault) {
             // the fused path needs another amount of scratch per query than a full row: its own chunking of the same region
-            int64_t fit = (int64_t)((region > 256 ? region - 256 : 0) / (coarse_mma_fused_bytes_per_query(ix->nlist) + qc_bytes));   // 256: alignment of the second part
+            int64_t fit = (int64_t)((region > 256 ? region - 256 : 0) / (coarse_mma_fused_bytes_per_query(ix->nlist, nprobe) + qc_bytes));   // 256: alignment of the second part
             if (fit >= 1) {
                 if (fit >= 128) fit -= fit % 128;   // whole query tiles of the tensor-core kernel
                 qchunk = fit < nq ? fit : nq;   // more queries per chunk than full rows would allow, or fewer

@@ -22,7 +22,7 @@
 //      decision with one warp per query and no block barrier.
 //
 //   Many clusters, few probes (nlist >= 8192, nprobe <= 64): the [queries][nlist] tile is never
-//   written.  A first pass runs the same kernel over the first quarter of the centroids only (at
+//   written.  A first pass runs the same kernel over the first quarter (few probes: eighth) of the centroids only (at
 //   most 4096; a random sample of the clusters: k-means was seeded with random points); probe_bound_kernel takes each
 //   query's nprobe-th smallest value of that sample, which is an upper bound of the nprobe-th
 //   smallest over all clusters, and adds twice the error bound; the main pass compares every
@@ -975,9 +975,13 @@ cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cuda
 constexpr int kSampleMax = 256 * kBoundPerThread;   // clusters of the bound-giving first pass, at most
 constexpr int kListCap = 1024;                      // candidate entries kept per query by the fused epilogue
 
-// Clusters of the first pass: a quarter of them (whole tiles), at most kSampleMax.
-static int sample_clusters(int nlist) {
+// Clusters of the first pass: a quarter of them (whole tiles, at most kSampleMax), or an eighth when
+// the list expected from that smaller sample (nlist * nprobe / sample) still stays within a quarter
+// of the list capacity (measured on 16 384 clusters, 32 probes: filtering 0.61 -> 0.56 ms).
+static int sample_clusters(int nlist, int nprobe) {
     int m = (nlist / 4) / kTileN * kTileN;
+    const int h = (nlist / 8) / kTileN * kTileN;
+    if (h >= 8 * kTileN && (int64_t)nlist * nprobe / h <= kListCap / 4) m = h;
     return m > kSampleMax ? kSampleMax : m;
 }
 
@@ -985,11 +989,11 @@ static int sample_clusters(int nlist) {
 // list (nlist * nprobe / sample, before the widening by the error bound) well under its capacity.
 bool coarse_mma_fused(int nlist, int nprobe) {
     if (nlist < 8192) return false;   // measured on 1024 clusters: 0.25 ms against 0.16 ms through full rows
-    return (int64_t)nlist * nprobe / sample_clusters(nlist) <= kListCap / 4;
+    return (int64_t)nlist * nprobe / sample_clusters(nlist, nprobe) <= kListCap / 4;
 }
 
 // Bytes of scratch per query of the fused path: sample row, cut, counter, candidate list.
-size_t coarse_mma_fused_bytes_per_query(int nlist) { return (size_t)sample_clusters(nlist) * 4 + 8 + (size_t)kListCap * 8; }
+size_t coarse_mma_fused_bytes_per_query(int nlist, int nprobe) { return (size_t)sample_clusters(nlist, nprobe) * 4 + 8 + (size_t)kListCap * 8; }
 
 // Tensor-core filtering of the queries [q0, q0 + nqc): returns cudaErrorNotSupported when the
 // tensor maps cannot be built (the caller then uses the plain kernels).  `tile` is scratch of at
@@ -1043,7 +1047,7 @@ cudaError_t launch_coarse_mma(const ivfpq_index* ix, const float* queries, int64
 
     if (fused) {   // the caller checked coarse_mma_fused() and sized the scratch for it
         // scratch: [nqc][sample] values | [nqc] cuts | [nqc] counters | [nqc][kListCap] (value, cluster)
-        const int nsample = sample_clusters(ix->nlist);
+        const int nsample = sample_clusters(ix->nlist, nprobe);
         float* sample = tile;
         float* cutp = sample + (size_t)nqc * nsample;
         int* ccount = reinterpret_cast<int*>(cutp + nqc);

@@ -137,7 +137,7 @@ bool rot_supported(int nsub, int dsub);
 bool coarse_mma_supported(int d, int nlist);
 size_t coarse_mma_derived_bytes(int nlist, int d, bool centered);
 bool coarse_mma_fused(int nlist, int nprobe);
-size_t coarse_mma_fused_bytes_per_query(int nlist);
+size_t coarse_mma_fused_bytes_per_query(int nlist, int nprobe);
 cudaError_t launch_entry_map(const ivfpq_index* ix, const uint8_t* codes, cudaStream_t st);
 cudaError_t launch_cnorm(const float* cent, int nlist, int d, float* cnorm, cudaStream_t st);
 cudaError_t launch_center(const float* cent, int nlist, int d, float* mu, float* cent_c, cudaStream_t st);
