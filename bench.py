@@ -42,9 +42,9 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per visited point of the dominant kernel
 # at the default settings of a workload, from the ncu capture summarised in the named file under
-# profiles/ (taken on a 1000-query batch: 7.304 GB for 475.8 M visited points; the traffic grows
+# profiles/ (taken on a 1000-query batch: 7.309 GB for 475.8 M visited points; the traffic grows
 # with the points visited).  An entry is dropped (traffic: null) when the kernel it describes changes.
-SCAN_DRAM_BYTES_PER_VISIT = {"c5": (15.35, "profiles/scan16x8_1024_c5_nq1000.md")}
+SCAN_DRAM_BYTES_PER_VISIT = {"c5": (15.36, "profiles/scan16x8_1024_c5_nq1000.md")}
 
 
 def log(*a):
